@@ -1,0 +1,174 @@
+/*
+ * matq.h — C ABI of the B200 (sm_100a) library for the nested
+ * int8 -> int4 -> int2 weight path of Matryoshka Quantization (MatQuant).
+ *
+ * Notation (the paper's): W is a weight matrix with N output channels (rows)
+ * and K input features, stored row-major as bf16; c = 8 is the width of the
+ * base code; r (1 <= r <= c) is the width sliced out of it; alpha and z are
+ * the per-output-channel scale and (real-valued) zero point of Eq. 1; x are
+ * bf16 activations; y are fp32 outputs.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers owned by the caller unless the comment says
+ *     "host".  The library never allocates, frees or keeps a pointer.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and
+ *     the call returns without synchronising.
+ *   - The return value is a status (MATQ_OK = 0).  Argument errors are found on
+ *     the host before anything is launched.  Errors that depend on the data
+ *     (non-finite weight, overflow list too small) are written by the kernels
+ *     into `dev_status` (device int32, nullable; first error wins; the caller
+ *     zeroes it) and never trap.
+ *   - 16-byte alignment of the matrix pointers and the row-length multiples
+ *     stated per call select the vectorised kernels; other shapes are either
+ *     served by slower generic kernels or rejected with MATQ_ERR_SHAPE /
+ *     MATQ_ERR_ALIGNMENT as stated.
+ *   - Thread-safe; no global mutable state.
+ */
+#ifndef MATQ_H_
+#define MATQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum matq_status {
+    MATQ_OK = 0,
+    MATQ_ERR_INVALID_ARG = 1,  /* null pointer, negative size, inconsistent optional arguments */
+    MATQ_ERR_UNSUPPORTED = 2,  /* c != 8, r outside [1, c], r not packable for this call */
+    MATQ_ERR_SHAPE = 3,        /* K (or ld*) is not a multiple the call requires */
+    MATQ_ERR_ALIGNMENT = 4,    /* pointer not aligned as the call requires */
+    MATQ_ERR_WORKSPACE = 5,    /* workspace missing or too small */
+    MATQ_ERR_CUDA = 6,         /* a CUDA runtime call failed (launch error, no sm_100 device) */
+    /* written to dev_status by kernels */
+    MATQ_ERR_NONFINITE = 8,    /* a weight is NaN or +-Inf */
+    MATQ_ERR_CAPACITY = 9,     /* extra-precision overflow list does not fit ovf_capacity */
+    MATQ_ERR_TIMEOUT = 10      /* a bounded device-side wait gave up */
+};
+
+/* Where matq_gemm_multi takes the weights from. */
+enum matq_src_kind {
+    MATQ_SRC_BF16 = 0,    /* bf16 W [N, K]; Eq. 1 is applied on the fly, alpha / zero are outputs */
+    MATQ_SRC_CODES8 = 1,  /* uint8 codes q [N, K]; alpha / zero are inputs */
+    MATQ_SRC_PACKED = 2   /* one packed r-bit plane (+ optional overflow list); n_r must be 1 */
+};
+
+/* matq_gemv flags */
+enum matq_gemv_flags {
+    MATQ_GEMV_AUTO = 0,        /* library picks the kernel */
+    MATQ_GEMV_CUDA_CORE = 1,   /* fp32 FMA path */
+    MATQ_GEMV_TENSOR = 2,      /* warp-level tensor-core path (bf16 x bf16 -> fp32) */
+    MATQ_GEMV_PATH_MASK = 0xff,
+    MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
+                                  fetching weights while the previous kernel in the stream drains and
+                                  waits for it only before reading x */
+};
+
+const char *matq_status_string(int status);
+int matq_version(void);
+
+/* Bytes per row of a packed r-bit plane: K * r / 8 for r in {8, 4, 2} and K a
+ * multiple of 8 / r; -1 otherwise. */
+int64_t matq_packed_row_bytes(int64_t K, int r);
+
+/*
+ * (1) MinMax quantisation, Eq. 1, one (alpha, z) per output channel:
+ *       alpha_n = (max_k W[n,k] - min_k W[n,k]) / (2^c - 1),  z_n = -min_k W[n,k] / alpha_n,
+ *       q[n,k]  = clamp(round_half_up(W[n,k] / alpha_n + z_n), 0, 2^c - 1)
+ *     evaluated in IEEE binary32, one correctly rounded operation per step in
+ *     the order written (true division, no fused multiply-add).  A constant row
+ *     gets alpha = 1, z = -W[n,0], codes 0.
+ *   W      in   bf16 [N, K], row stride ldw elements (ldw >= K)
+ *   q      out  uint8 [N, K] contiguous; may be NULL when only alpha / zero are wanted
+ *   alpha  out  fp32 [N]
+ *   zero   out  fp32 [N]
+ *   A NaN / Inf weight sets dev_status = MATQ_ERR_NONFINITE; that row's outputs are unspecified.
+ *   Fast path: W and q 16-byte aligned, K % 16 == 0, ldw % 8 == 0, K <= 65536.  Any other
+ *   shape runs a scalar kernel.  c must be 8.
+ */
+int matq_quantize(const void *W, int64_t N, int64_t K, int64_t ldw, int c,
+                  uint8_t *q, float *alpha, float *zero,
+                  int32_t *dev_status, void *stream);
+
+/*
+ * (2) MSB slicing S(q, r) of Eq. 6 (extra_precision = 0) or of the Errata's
+ *     Eq. 8 (extra_precision = 1), then packing.  With sh = c - r:
+ *       k      = min((q + 2^(sh-1)) >> sh, 2^r - 1)      (k = q when sh = 0)
+ *       S(q,r) = k << sh
+ *     Plane format: for r in {8, 4, 2}, byte j of a row holds the fields k of
+ *     elements j*(8/r) + i, i = 0 .. 8/r - 1, field i in bits [i*r, (i+1)*r).
+ *     Rows are contiguous, K*r/8 bytes each.  Slices are always taken from the
+ *     c-bit code (Section 3.2), never from another slice.
+ *   q                in   uint8 [N, K] contiguous
+ *   packed           out  uint8 [N, K*r/8]; NULL allowed (then only the other outputs are written);
+ *                         non-NULL requires r in {8, 4, 2} and K % (8/r) == 0
+ *   sliced_unpacked  out  uint8 [N, K] = S(q, r) of Eq. 6, any 1 <= r <= 8; NULL allowed
+ *   Extra precision (Eq. 8 keeps bucket 2^r): the plane holds the CLAMPED field,
+ *   so it is byte-identical to the standard plane, and the elements whose Eq. 8
+ *   value is one bucket higher (exactly those with q >= 2^c - 2^(sh-1)) are listed:
+ *   ovf_row_ptr      out  int32 [N + 1]; row n's entries are ovf_col[ovf_row_ptr[n] .. ovf_row_ptr[n+1])
+ *   ovf_col          out  uint16 [ovf_capacity] column indices, ascending within a row (needs K <= 65536)
+ *   ovf_count        out  int64 [1] (device): total number of overflow elements, written even when
+ *                         it exceeds ovf_capacity; then dev_status = MATQ_ERR_CAPACITY and ovf_col is unspecified
+ *   All three are required iff extra_precision != 0 and r < c; otherwise they are ignored
+ *   (ovf_count, if non-NULL, is set to 0).  The result is deterministic.
+ */
+int matq_slice_pack(const uint8_t *q, int64_t N, int64_t K, int c, int r, int extra_precision,
+                    uint8_t *packed, uint8_t *sliced_unpacked,
+                    int32_t *ovf_row_ptr, uint16_t *ovf_col, int64_t ovf_capacity, int64_t *ovf_count,
+                    int32_t *dev_status, void *stream);
+
+/*
+ * (3) Decode-time weight-only quantised linear layer on a packed r-bit plane:
+ *       y[b,n] = sum_k x[b,k] * alpha_n * (S[n,k] - z_n),   S = k << (c - r)
+ *     (dequantisation alpha * (S - z) with the same alpha, z at every r, since
+ *     Eq. 6 returns values on the c-bit grid).  When the overflow list is given,
+ *     S[n,j] is one bucket (2^(c-r)) higher at the listed columns j (Eq. 8).
+ *   packed       in   uint8 [N, K*r/8], r in {8, 4, 2}, 16-byte aligned, K % 128 == 0
+ *   alpha, zero  in   fp32 [N]
+ *   ovf_row_ptr, ovf_col  in   both NULL or both given (format as in matq_slice_pack)
+ *   x            in   bf16 [B, K], row stride ldx elements, 1 <= B <= 16, 16-byte aligned, ldx % 8 == 0
+ *   y            out  fp32 [B, N], row stride ldy elements
+ *   workspace         device scratch of at least matq_gemv_workspace_bytes(...) bytes (may be NULL if that is 0)
+ *   flags             matq_gemv_flags
+ *   fp32 accumulation; results differ from an fp64 evaluation by rounding only.
+ */
+size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B);
+int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
+              const float *alpha, const float *zero,
+              const int32_t *ovf_row_ptr, const uint16_t *ovf_col,
+              const void *x, int B, int64_t ldx, float *y, int64_t ldy,
+              void *workspace, size_t workspace_bytes, unsigned flags,
+              int32_t *dev_status, void *stream);
+
+/*
+ * (4) Multi-precision dense forward of MatQuant co-training (Eq. 7): for every
+ *     r in rs, Y_r = X . dequant(S(Q(W, c), r))^T, all precisions from one pass
+ *     over the weights.  The integer fields enter the tensor cores exactly as
+ *     bf16 (0 .. 255 are exact) with fp32 accumulation; alpha and z * sum_k x
+ *     are applied per channel afterwards:
+ *       Y_r[m,n] = alpha_n * ( 2^(c-r) * sum_k X[m,k] k_r[n,k]  -  z_n * sum_k X[m,k] ).
+ *   Wsrc         in   per src_kind (matq_src_kind)
+ *   alpha, zero  out for MATQ_SRC_BF16, in otherwise; fp32 [N]
+ *   extra_precision   slice with Eq. 8 instead of Eq. 6 (for MATQ_SRC_PACKED: apply the overflow list)
+ *   X            in   bf16 [M, K], row stride ldx
+ *   rs           in   HOST array of n_r distinct precisions (1 <= n_r <= 3), e.g. {8, 4, 2}
+ *   Y            in   HOST array of n_r device pointers, each fp32 [M, N] with row stride ldy
+ *   workspace         device scratch of at least matq_gemm_multi_workspace_bytes(...) bytes
+ *   Requires K % 64 == 0, N % 8 == 0, 16-byte aligned pointers.
+ */
+size_t matq_gemm_multi_workspace_bytes(int src_kind, int64_t M, int64_t N, int64_t K, int n_r);
+int matq_gemm_multi(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
+                    float *alpha, float *zero, int extra_precision,
+                    const int32_t *ovf_row_ptr, const uint16_t *ovf_col,
+                    const void *X, int64_t M, int64_t ldx,
+                    const int *rs, int n_r, float *const *Y, int64_t ldy,
+                    void *workspace, size_t workspace_bytes,
+                    int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MATQ_H_ */

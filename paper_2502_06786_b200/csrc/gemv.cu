@@ -1,0 +1,33 @@
+// matq_gemv: host-side validation and kernel selection for the decode GEMV.
+#include "common.cuh"
+#include "gemv_cuda_core.cuh"
+
+extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
+    (void)N; (void)K; (void)r; (void)B;
+    return 0;   // the K-split is reduced inside warps / CTAs; no scratch is needed
+}
+
+extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int r,
+                         const float* alpha, const float* zero,
+                         const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
+                         const void* x, int B, int64_t ldx, float* y, int64_t ldy,
+                         void* workspace, size_t workspace_bytes, unsigned flags,
+                         int32_t* dev_status, void* stream) {
+    using namespace matq;
+    (void)workspace; (void)workspace_bytes; (void)dev_status;
+    if (!packed || !alpha || !zero || !x || !y || N < 0 || K <= 0 || B < 1 || B > 16) return MATQ_ERR_INVALID_ARG;
+    if ((ovf_row_ptr == nullptr) != (ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
+    if (c != kCodeBits || !(r == 8 || r == 4 || r == 2)) return MATQ_ERR_UNSUPPORTED;
+    if (K % 128 != 0 || ldx < K || ldx % 8 != 0 || ldy < N) return MATQ_ERR_SHAPE;
+    if (ovf_row_ptr && K > 65536) return MATQ_ERR_SHAPE;
+    if (!aligned16(packed) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
+    const unsigned path = flags & MATQ_GEMV_PATH_MASK;
+    if (path > MATQ_GEMV_TENSOR || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
+    if (N == 0) return MATQ_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
+    if (r == 8) launch_gemv_cuda_core<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+    else if (r == 4) launch_gemv_cuda_core<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+    else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+    return launch_status();
+}

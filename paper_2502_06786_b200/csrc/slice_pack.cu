@@ -1,0 +1,263 @@
+// matq_slice_pack: MSB slicing S(q, r) (Eq. 6), the un-clamped variant of the
+// Errata (Eq. 8) as a sparse overflow list, and packing into r-bit planes.
+//
+// The pass is pure integer work bound by HBM: 1 byte read and r/8 bytes written
+// per weight.  Four codes are sliced at once inside a 32-bit register:
+//   a = (w >> sh) & fieldmask        top r bits of every byte
+//   b = (w >> (sh-1)) & 0x01010101   the (r+1)-th most significant bit (Appendix A's rounding bit)
+//   s = a + b                        <= 2^r per byte, never carries across bytes
+//   ov = (s >> r) & 0x01010101       1 where rounding overflowed into bucket 2^r
+//   k = s - ov                       the clamp of Eq. 6
+// `ov` is exactly the extra bucket Eq. 8 keeps, so the extra-precision list is
+// a by-product of the same arithmetic.
+//
+// Extra precision takes three stream-ordered kernels: (1) pack + per-row
+// overflow counts, (2) one-block exclusive scan of the counts into
+// ovf_row_ptr, (3) one warp per row re-reads the codes and writes the
+// ascending column list at its row's offset.
+#include "common.cuh"
+
+namespace matq {
+namespace {
+
+constexpr int kSliceThreads = 256;
+
+struct Sliced {
+    uint32_t k;   // four r-bit fields, one per byte
+    uint32_t ov;  // bit 0 of each byte: Eq. 8 differs from Eq. 6 here
+};
+
+__device__ __forceinline__ Sliced slice4(uint32_t w, int r) {
+    const int sh = kCodeBits - r;
+    if (sh == 0) return {w, 0u};
+    const uint32_t fieldmask = 0x01010101u * ((1u << r) - 1u);
+    const uint32_t a = (w >> sh) & fieldmask;
+    const uint32_t b = (w >> (sh - 1)) & 0x01010101u;
+    const uint32_t s = a + b;
+    const uint32_t ov = (s >> r) & 0x01010101u;
+    return {s - ov, ov};
+}
+
+// Four one-byte fields -> 4*R contiguous bits, element 0 in the least significant bits.
+template <int R>
+__device__ __forceinline__ uint32_t pack4(uint32_t k) {
+    if (R == 8) return k;
+    if (R == 4) {
+        const uint32_t t = (k | (k >> 4)) & 0x00ff00ffu;
+        return (t | (t >> 8)) & 0xffffu;
+    }
+    const uint32_t t = (k | (k >> 6)) & 0x000f000fu;   // R == 2
+    return (t | (t >> 12)) & 0xffu;
+}
+
+// bits 0, 8, 16, 24 -> bits 0..3
+__device__ __forceinline__ uint32_t gather_byte_lsbs(uint32_t ov) { return ((ov * 0x01020408u) >> 24) & 0xfu; }
+
+// Fast path: K % 16 == 0 and 16-byte aligned buffers.  One thread = 16 codes.
+// PACK_R = 0: no packed output (any r, runtime); otherwise r == PACK_R.
+template <int PACK_R>
+__global__ void __launch_bounds__(kSliceThreads)
+slice_pack_vec(const uint4* __restrict__ q, int64_t nchunks, int chunks_per_row, int r_runtime,
+               uint8_t* __restrict__ packed, uint4* __restrict__ sliced, int32_t* __restrict__ row_count) {
+    const int r = PACK_R ? PACK_R : r_runtime;
+    const int sh = kCodeBits - r;
+    const int64_t stride = (int64_t)gridDim.x * kSliceThreads;
+    for (int64_t i = (int64_t)blockIdx.x * kSliceThreads + threadIdx.x; i < nchunks; i += stride) {
+        const uint4 v = ld_stream_u4(q + i);
+        const Sliced s0 = slice4(v.x, r), s1 = slice4(v.y, r), s2 = slice4(v.z, r), s3 = slice4(v.w, r);
+        if (PACK_R == 8) {
+            reinterpret_cast<uint4*>(packed)[i] = make_uint4(s0.k, s1.k, s2.k, s3.k);
+        } else if (PACK_R == 4) {
+            reinterpret_cast<uint2*>(packed)[i] =
+                make_uint2(pack4<4>(s0.k) | (pack4<4>(s1.k) << 16), pack4<4>(s2.k) | (pack4<4>(s3.k) << 16));
+        } else if (PACK_R == 2) {
+            reinterpret_cast<uint32_t*>(packed)[i] =
+                pack4<2>(s0.k) | (pack4<2>(s1.k) << 8) | (pack4<2>(s2.k) << 16) | (pack4<2>(s3.k) << 24);
+        }
+        if (sliced) sliced[i] = make_uint4(s0.k << sh, s1.k << sh, s2.k << sh, s3.k << sh);
+        if (row_count) {
+            const int cnt = __popc(s0.ov) + __popc(s1.ov) + __popc(s2.ov) + __popc(s3.ov);
+            if (cnt) atomicAdd(row_count + (i / chunks_per_row), cnt);
+        }
+    }
+}
+
+// Any K / alignment: one thread = the codes of one packed byte (or one code when nothing is packed).
+__global__ void __launch_bounds__(kSliceThreads)
+slice_pack_generic(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, int per_byte,
+                   uint8_t* __restrict__ packed, uint8_t* __restrict__ sliced, int32_t* __restrict__ row_count) {
+    const int sh = kCodeBits - r;
+    const int64_t groups = N * K / per_byte;
+    const int64_t stride = (int64_t)gridDim.x * kSliceThreads;
+    for (int64_t g = (int64_t)blockIdx.x * kSliceThreads + threadIdx.x; g < groups; g += stride) {
+        uint32_t byte = 0;
+        for (int i = 0; i < per_byte; ++i) {
+            const int64_t e = g * per_byte + i;
+            const Sliced s = slice4(q[e], r);
+            byte |= (s.k & 0xffu) << (i * r);
+            if (sliced) sliced[e] = (uint8_t)((s.k & 0xffu) << sh);
+            if (row_count && (s.ov & 1u)) atomicAdd(row_count + e / K, 1);
+        }
+        if (packed) packed[g] = (uint8_t)byte;
+    }
+}
+
+// row_ptr[n+1] holds row n's count on entry; on exit row_ptr is the exclusive scan.
+__global__ void __launch_bounds__(1024)
+ovf_scan(int32_t* __restrict__ row_ptr, int64_t N, int64_t capacity, int64_t* __restrict__ total_out,
+         int32_t* dev_status) {
+    __shared__ int64_t warp_sum[32];
+    __shared__ int64_t carry_s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { carry_s = 0; row_ptr[0] = 0; }
+    __syncthreads();
+    for (int64_t base = 0; base < N; base += 1024) {
+        const int64_t n = base + threadIdx.x;
+        int64_t v = (n < N) ? row_ptr[n + 1] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int64_t t = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += t;
+        }
+        if (lane == 31) warp_sum[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            int64_t w = warp_sum[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int64_t t = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += t;
+            }
+            warp_sum[lane] = w;
+        }
+        __syncthreads();
+        const int64_t carry = carry_s;
+        const int64_t incl = carry + v + (warp ? warp_sum[warp - 1] : 0);
+        if (n < N) row_ptr[n + 1] = (int32_t)(incl > 0x7fffffff ? 0x7fffffff : incl);
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const int64_t total = carry_s;
+        *total_out = total;
+        if (total > capacity || total > 0x7fffffff) report(dev_status, MATQ_ERR_CAPACITY);
+    }
+}
+
+// One warp per row writes the ascending column indices of the overflow elements.
+template <bool VEC>
+__global__ void __launch_bounds__(kSliceThreads)
+ovf_fill(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, const int32_t* __restrict__ row_ptr,
+         const int64_t* __restrict__ total, int64_t capacity, uint16_t* __restrict__ ovf_col) {
+    if (*total > capacity || *total > 0x7fffffff) return;   // lists are unspecified in that case
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (kSliceThreads / 32);
+    constexpr int kPerLane = VEC ? 16 : 1;
+    for (int64_t n = (int64_t)blockIdx.x * (kSliceThreads / 32) + (threadIdx.x >> 5); n < N; n += warps) {
+        int64_t out = row_ptr[n];
+        if (row_ptr[n + 1] == out) continue;
+        const uint8_t* row = q + n * K;
+        for (int64_t k0 = 0; k0 < K; k0 += 32 * kPerLane) {
+            const int64_t k = k0 + (int64_t)lane * kPerLane;
+            uint32_t mask = 0;
+            if (k < K) {
+                if (VEC) {
+                    const uint4 v = ld_stream_u4(row + k);
+                    mask = gather_byte_lsbs(slice4(v.x, r).ov) | (gather_byte_lsbs(slice4(v.y, r).ov) << 4) |
+                           (gather_byte_lsbs(slice4(v.z, r).ov) << 8) | (gather_byte_lsbs(slice4(v.w, r).ov) << 12);
+                } else {
+                    mask = slice4(row[k], r).ov & 1u;
+                }
+            }
+            const int cnt = __popc(mask);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            int64_t pos = out + incl - cnt;
+            while (mask) {
+                const int b = __ffs(mask) - 1;
+                ovf_col[pos++] = (uint16_t)(k + b);
+                mask &= mask - 1;
+            }
+            out += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+}
+
+template <int PACK_R>
+void launch_vec(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, uint8_t* sliced,
+                int32_t* row_count, cudaStream_t s) {
+    const int64_t nchunks = N * K / 16;
+    int64_t blocks = (nchunks + kSliceThreads - 1) / kSliceThreads;
+    const int64_t cap = (int64_t)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    slice_pack_vec<PACK_R><<<(unsigned)blocks, kSliceThreads, 0, s>>>(
+        reinterpret_cast<const uint4*>(q), nchunks, (int)(K / 16), r, packed, reinterpret_cast<uint4*>(sliced), row_count);
+}
+
+}  // namespace
+}  // namespace matq
+
+extern "C" int64_t matq_packed_row_bytes(int64_t K, int r) {
+    if (!(r == 8 || r == 4 || r == 2) || K <= 0 || (K % (8 / r)) != 0) return -1;
+    return K * r / 8;
+}
+
+extern "C" int matq_slice_pack(const uint8_t* q, int64_t N, int64_t K, int c, int r, int extra_precision,
+                               uint8_t* packed, uint8_t* sliced_unpacked,
+                               int32_t* ovf_row_ptr, uint16_t* ovf_col, int64_t ovf_capacity, int64_t* ovf_count,
+                               int32_t* dev_status, void* stream) {
+    using namespace matq;
+    if (!q || N < 0 || K <= 0) return MATQ_ERR_INVALID_ARG;
+    if (c != kCodeBits || r < 1 || r > c) return MATQ_ERR_UNSUPPORTED;
+    const bool packable = (r == 8 || r == 4 || r == 2);
+    if (packed && !packable) return MATQ_ERR_UNSUPPORTED;
+    const int per_byte = packed ? 8 / r : 1;
+    if (packed && (K % per_byte) != 0) return MATQ_ERR_SHAPE;
+    const bool want_ovf = extra_precision && r < c;
+    if (want_ovf && (!ovf_row_ptr || !ovf_col || !ovf_count || ovf_capacity < 0)) return MATQ_ERR_INVALID_ARG;
+    if (want_ovf && K > 65536) return MATQ_ERR_SHAPE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!want_ovf && ovf_count && cudaMemsetAsync(ovf_count, 0, sizeof(int64_t), s) != cudaSuccess) return MATQ_ERR_CUDA;
+    if (N == 0) {
+        if (want_ovf && (cudaMemsetAsync(ovf_row_ptr, 0, sizeof(int32_t), s) != cudaSuccess ||
+                         cudaMemsetAsync(ovf_count, 0, sizeof(int64_t), s) != cudaSuccess)) return MATQ_ERR_CUDA;
+        return MATQ_OK;
+    }
+    int32_t* row_count = nullptr;
+    if (want_ovf) {
+        if (cudaMemsetAsync(ovf_row_ptr, 0, (size_t)(N + 1) * sizeof(int32_t), s) != cudaSuccess) return MATQ_ERR_CUDA;
+        row_count = ovf_row_ptr + 1;
+    }
+    const bool vec = (K % 16 == 0) && aligned16(q) && (!packed || aligned16(packed)) &&
+                     (!sliced_unpacked || aligned16(sliced_unpacked));
+    if (packed || sliced_unpacked || row_count) {
+        if (vec) {
+            if (!packed) launch_vec<0>(q, N, K, r, packed, sliced_unpacked, row_count, s);
+            else if (r == 8) launch_vec<8>(q, N, K, r, packed, sliced_unpacked, row_count, s);
+            else if (r == 4) launch_vec<4>(q, N, K, r, packed, sliced_unpacked, row_count, s);
+            else launch_vec<2>(q, N, K, r, packed, sliced_unpacked, row_count, s);
+        } else {
+            const int64_t groups = N * K / per_byte;
+            int64_t blocks = (groups + kSliceThreads - 1) / kSliceThreads;
+            const int64_t cap = (int64_t)sm_count() * 32;
+            if (blocks > cap) blocks = cap;
+            slice_pack_generic<<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, per_byte, packed, sliced_unpacked, row_count);
+        }
+        if (launch_status() != MATQ_OK) return MATQ_ERR_CUDA;
+    }
+    if (want_ovf) {
+        ovf_scan<<<1, 1024, 0, s>>>(ovf_row_ptr, N, ovf_capacity, ovf_count, dev_status);
+        const int warps_per_block = kSliceThreads / 32;
+        int64_t blocks = (N + warps_per_block - 1) / warps_per_block;
+        const int64_t cap = (int64_t)sm_count() * 32;
+        if (blocks > cap) blocks = cap;
+        if (vec) ovf_fill<true><<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
+        else ovf_fill<false><<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
+    }
+    return launch_status();
+}
