@@ -1,0 +1,205 @@
+"""GPU parity: every CUDA entry point against the CPU oracle on the same seeded inputs.
+
+Integer outputs (codes, slices, packed bytes, overflow lists) must match bit
+for bit; alpha and z must be equal as fp32 values; y must satisfy
+max|dy| <= 1e-3 * rms(y_oracle) on the fp32 FMA path.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2502_06786_b200 import binding as mq
+from paper_2502_06786_b200 import synth
+from tests.util import bf16_dev, dev, host, rms, status_word
+
+pytestmark = pytest.mark.gpu
+
+TOL_FMA = 1e-3
+
+
+# ------------------------------------------------------------------ quantize
+
+@pytest.mark.parametrize("N,K,dist", [(1, 16, "normal"), (37, 1024, "normal"), (300, 2304, "normal"),
+                                      (64, 4096, "student"), (5, 14336, "normal"), (19, 1000, "normal"),
+                                      (7, 24, "student"), (3, 65536, "normal")])
+def test_quantize_bit_exact(N, K, dist):
+    W = synth.normal_bf16((N, K), 0.02, 100 + N) if dist == "normal" else synth.student_t_bf16((N, K), 3.0, 0.02, 200 + N)
+    st, q_ref, a_ref, z_ref = ref.quantize(W)
+    assert st == ref.OK
+    status = status_word()
+    q, a, z = mq.quantize(bf16_dev(W), dev_status=status)
+    assert np.array_equal(host(q), q_ref)
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert int(host(status)[0]) == mq.OK
+
+
+def test_quantize_special_rows_and_strided_input():
+    K = 256
+    W = synth.normal_bf16((6, K), 0.02, 7)
+    Wf = synth.bf16_bits_to_f32(W).copy()
+    Wf[1, :] = 0.375                      # constant row: alpha = 1, z = -0.375, codes 0
+    Wf[2, :] = np.abs(Wf[2, :]) + 1.0     # same-sign row: z < 0
+    Wf[3, :] = 0.0                        # all-zero row
+    Wf[4, :8] = [0.0, 255.0, 0.5, 1.5, 2.5, 126.5, 3.25, 17.75]   # alpha = 1 ties round up
+    Wf[4, 8:] = 1.0
+    W = synth.f32_to_bf16_bits(Wf)
+    st, q_ref, a_ref, z_ref = ref.quantize(W)
+    q, a, z = mq.quantize(bf16_dev(W))
+    assert np.array_equal(host(q), q_ref) and np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert host(q)[4, :8].tolist() == [0, 255, 1, 2, 3, 127, 3, 18]
+    # row stride larger than K (a view into a wider matrix), and alpha / z only
+    wide = torch.zeros((6, K + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :K] = bf16_dev(W)
+    q2, a2, z2 = mq.quantize(wide[:, :K])
+    assert np.array_equal(host(q2), q_ref) and np.array_equal(host(a2), a_ref)
+    q3, a3, z3 = mq.quantize(bf16_dev(W), want_codes=False)
+    assert q3 is None and np.array_equal(host(a3), a_ref) and np.array_equal(host(z3), z_ref)
+
+
+def test_quantize_reports_nonfinite_without_trapping():
+    Wf = synth.bf16_bits_to_f32(synth.normal_bf16((4, 128), 0.02, 9)).copy()
+    Wf[2, 77] = np.inf
+    status = status_word()
+    mq.quantize(bf16_dev(synth.f32_to_bf16_bits(Wf)), dev_status=status)
+    assert int(host(status)[0]) == mq.ERR_NONFINITE
+    Wf[2, 77] = np.nan
+    status = status_word()
+    mq.quantize(bf16_dev(synth.f32_to_bf16_bits(Wf)), dev_status=status)
+    assert int(host(status)[0]) == mq.ERR_NONFINITE
+    # the context is still usable
+    q, a, z = mq.quantize(bf16_dev(synth.normal_bf16((4, 128), 0.02, 9)))
+    assert host(q).shape == (4, 128)
+
+
+# ---------------------------------------------------------------- slice/pack
+
+@pytest.mark.parametrize("r", range(1, 9))
+def test_slice_all_256_codes_every_r(r):
+    q = np.tile(np.arange(256, dtype=np.uint8), (3, 1))
+    out = mq.slice_pack(dev(q), r, want_packed=False, want_unpacked=True)
+    _, S = ref.slice_values(q, r)
+    assert np.array_equal(host(out["sliced"]).astype(np.uint16), S)
+
+
+@pytest.mark.parametrize("r", [8, 4, 2])
+@pytest.mark.parametrize("N,K", [(1, 16), (33, 2304), (129, 4096), (7, 1000), (5, 24), (0, 64)])
+def test_pack_bit_exact(r, N, K):
+    q = synth.uniform_codes((N, K), 300 + N + r)
+    out = mq.slice_pack(dev(q), r, want_unpacked=True)
+    want = ref.slice_pack(q, r)
+    assert want["status"] == ref.OK
+    assert np.array_equal(host(out["packed"]), want["packed"])
+    assert np.array_equal(host(out["sliced"]), want["sliced"])
+
+
+@pytest.mark.parametrize("r", [4, 2])
+@pytest.mark.parametrize("N,K,p", [(64, 2304, 0.05), (1500, 512, 0.125), (9, 1000, 0.3), (40, 4096, 0.0)])
+def test_extra_precision_lists_bit_exact(r, N, K, p):
+    q = synth.skewed_codes((N, K), p, 224, 400 + N) if p > 0 else synth.uniform_codes((N, K), 1) // 2
+    if N > 8:
+        q[3, :] = 255     # a full row
+        q[5, :] = 0       # an empty row
+    status = status_word()
+    out = mq.slice_pack(dev(q), r, extra_precision=True, dev_status=status)
+    want = ref.slice_pack(q, r, extra_precision=True)
+    cnt = int(host(out["ovf_count"])[0])
+    assert cnt == want["ovf_count"]
+    assert np.array_equal(host(out["packed"]), want["packed"])
+    assert np.array_equal(host(out["ovf_row_ptr"]), want["ovf_row_ptr"])
+    assert np.array_equal(host(out["ovf_col"])[:cnt], want["ovf_col"])
+    assert int(host(status)[0]) == mq.OK
+    # standard plane == E.P. base plane
+    std = mq.slice_pack(dev(q), r)
+    assert torch.equal(std["packed"], out["packed"])
+
+
+def test_extra_precision_capacity_error_is_a_status():
+    q = synth.skewed_codes((32, 512), 0.2, 224, 77)
+    want = ref.slice_pack(q, 2, extra_precision=True)
+    status = status_word()
+    out = mq.slice_pack(dev(q), 2, extra_precision=True, ovf_capacity=16, dev_status=status)
+    assert int(host(out["ovf_count"])[0]) == want["ovf_count"] > 16
+    assert int(host(status)[0]) == mq.ERR_CAPACITY
+    assert np.array_equal(host(out["ovf_row_ptr"]), want["ovf_row_ptr"])
+    # r = c: no overflow, count forced to 0
+    cnt = torch.full((1,), 5, dtype=torch.int64, device="cuda")
+    mq.slice_pack(dev(q), 8, extra_precision=True, ovf_count=cnt)
+    assert int(host(cnt)[0]) == 0
+
+
+# ---------------------------------------------------------------------- gemv
+
+def _gemv_case(N, K, B, r, seed, ep=False, flags=0):
+    W = synth.normal_bf16((N, K), 0.02, seed)
+    st, q, a, z = ref.quantize(W)
+    if ep:
+        q = synth.skewed_codes((N, K), 0.05, 224, seed + 5)
+    x = synth.normal_bf16((B, K), 1.0, seed + 1)
+    sp = ref.slice_pack(q, r, extra_precision=ep)
+    rp = sp["ovf_row_ptr"] if ep else None
+    col = sp["ovf_col"] if ep else None
+    st, y_ref = ref.gemv(sp["packed"], K, r, a, z, x, rp, col)
+    assert st == ref.OK
+    y = mq.gemv(dev(sp["packed"]), K, r, dev(a), dev(z), bf16_dev(x),
+                ovf_row_ptr=dev(rp) if ep else None,
+                ovf_col=dev(col if col.size else np.zeros(1, np.uint16)) if ep else None, flags=flags)
+    return host(y), y_ref
+
+
+@pytest.mark.parametrize("r", [8, 4, 2])
+@pytest.mark.parametrize("N,K,B", [(1024, 1024, 1), (300, 2304, 1), (130, 9216, 8), (77, 3584, 4), (3, 128, 16),
+                                   (257, 14336, 3), (64, 256, 5)])
+def test_gemv_cuda_core_within_tolerance(r, N, K, B):
+    y, y_ref = _gemv_case(N, K, B, r, 500 + N + r, flags=mq.GEMV_CUDA_CORE)
+    assert np.abs(y - y_ref).max() <= TOL_FMA * rms(y_ref)
+
+
+@pytest.mark.parametrize("r", [4, 2])
+@pytest.mark.parametrize("B", [1, 8])
+def test_gemv_extra_precision(r, B):
+    y, y_ref = _gemv_case(130, 2304, B, r, 600 + r, ep=True, flags=mq.GEMV_CUDA_CORE)
+    assert np.abs(y - y_ref).max() <= TOL_FMA * rms(y_ref)
+
+
+@pytest.mark.parametrize("r", [8, 4, 2])
+def test_gemv_exact_integer_case(r):
+    # alpha = 1, z = 0, integer x: every partial sum is an exact fp32 integer, so the result must be exact.
+    N, K, B = 70, 512, 4
+    q = synth.uniform_codes((N, K), 700 + r)
+    x = synth.small_int_bf16((B, K), -4, 4, 701)
+    a = np.ones(N, np.float32); z = np.zeros(N, np.float32)
+    sp = ref.slice_pack(q, r)
+    _, y_ref = ref.gemv(sp["packed"], K, r, a, z, x)
+    y = mq.gemv(dev(sp["packed"]), K, r, dev(a), dev(z), bf16_dev(x), flags=mq.GEMV_CUDA_CORE)
+    assert np.array_equal(host(y).astype(np.float64), y_ref)
+
+
+def test_gemv_strided_x_and_y():
+    N, K, B, r = 50, 256, 3, 4
+    q = synth.uniform_codes((N, K), 800)
+    a = np.full(N, 0.01, np.float32); z = np.full(N, 100.0, np.float32)
+    x = synth.normal_bf16((B, K), 1.0, 801)
+    sp = ref.slice_pack(q, r)
+    _, y_ref = ref.gemv(sp["packed"], K, r, a, z, x)
+    xw = torch.zeros((B, K + 8), dtype=torch.bfloat16, device="cuda"); xw[:, :K] = bf16_dev(x)
+    yw = torch.full((B, N + 5), -1.0, dtype=torch.float32, device="cuda")
+    mq.gemv(dev(sp["packed"]), K, r, dev(a), dev(z), xw[:, :K], y=yw[:, :N])
+    assert np.abs(host(yw)[:, :N] - y_ref).max() <= TOL_FMA * rms(y_ref)
+    assert np.all(host(yw)[:, N:] == -1.0)
+
+
+def test_full_path_quantize_slice_pack_gemv():
+    # bf16 weights -> codes -> plane -> y, everything on the GPU, against the oracle end to end.
+    N, K, B = 260, 2304, 2
+    W = synth.normal_bf16((N, K), 0.02, 900)
+    x = synth.normal_bf16((B, K), 1.0, 901)
+    q, a, z = mq.quantize(bf16_dev(W))
+    st, q_ref, a_ref, z_ref = ref.quantize(W)
+    for r in (8, 4, 2):
+        sp = mq.slice_pack(q, r)
+        y = mq.gemv(sp["packed"], K, r, a, z, bf16_dev(x))
+        spr = ref.slice_pack(q_ref, r)
+        _, y_ref = ref.gemv(spr["packed"], K, r, a_ref, z_ref, x)
+        assert np.array_equal(host(sp["packed"]), spr["packed"])
+        assert np.abs(host(y) - y_ref).max() <= TOL_FMA * rms(y_ref)
