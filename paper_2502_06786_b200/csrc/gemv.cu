@@ -15,12 +15,12 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
                          int32_t* dev_status, void* stream) {
     using namespace matq;
     (void)workspace; (void)workspace_bytes; (void)dev_status;
-    if (!packed || !alpha || !zero || !x || !y || N < 0 || K <= 0 || B < 1 || B > 16) return MATQ_ERR_INVALID_ARG;
+    if (N < 0 || K <= 0 || B < 1 || B > 16 || !x || (N > 0 && (!packed || !alpha || !zero || !y))) return MATQ_ERR_INVALID_ARG;
     if ((ovf_row_ptr == nullptr) != (ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits || !(r == 8 || r == 4 || r == 2)) return MATQ_ERR_UNSUPPORTED;
     if (K % 128 != 0 || ldx < K || ldx % 8 != 0 || ldy < N) return MATQ_ERR_SHAPE;
     if (ovf_row_ptr && K > 65536) return MATQ_ERR_SHAPE;
-    if (!aligned16(packed) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
+    if ((N > 0 && !aligned16(packed)) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
     const unsigned path = flags & MATQ_GEMV_PATH_MASK;
     if (path > MATQ_GEMV_TENSOR || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
     if (N == 0) return MATQ_OK;

@@ -157,7 +157,7 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
                              uint8_t* q, float* alpha, float* zero,
                              int32_t* dev_status, void* stream) {
     using namespace matq;
-    if (!W || !alpha || !zero || N < 0 || K <= 0 || ldw < K) return MATQ_ERR_INVALID_ARG;
+    if (N < 0 || K <= 0 || ldw < K || (N > 0 && (!W || !alpha || !zero))) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

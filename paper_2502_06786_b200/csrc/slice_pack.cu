@@ -212,7 +212,7 @@ extern "C" int matq_slice_pack(const uint8_t* q, int64_t N, int64_t K, int c, in
                                int32_t* ovf_row_ptr, uint16_t* ovf_col, int64_t ovf_capacity, int64_t* ovf_count,
                                int32_t* dev_status, void* stream) {
     using namespace matq;
-    if (!q || N < 0 || K <= 0) return MATQ_ERR_INVALID_ARG;
+    if (N < 0 || K <= 0 || (!q && N > 0)) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits || r < 1 || r > c) return MATQ_ERR_UNSUPPORTED;
     const bool packable = (r == 8 || r == 4 || r == 2);
     if (packed && !packable) return MATQ_ERR_UNSUPPORTED;
