@@ -1,6 +1,7 @@
 // matq_gemv: host-side validation and kernel selection for the decode GEMV.
 #include "common.cuh"
 #include "gemv_cuda_core.cuh"
+#include "gemv_tensor.cuh"
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
     (void)N; (void)K; (void)r; (void)B;
@@ -26,8 +27,17 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
-    if (r == 8) launch_gemv_cuda_core<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
-    else if (r == 4) launch_gemv_cuda_core<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
-    else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+    if (path == MATQ_GEMV_CUDA_CORE) {
+        if (r == 8) launch_gemv_cuda_core<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        else if (r == 4) launch_gemv_cuda_core<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        return launch_status();
+    }
+    int st;
+#define MATQ_GEMV_T(RR, NT) launch_gemv_tensor<RR, 2, NT, 4, 2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+    if (B <= 8) st = (r == 8) ? MATQ_GEMV_T(8, 1) : (r == 4) ? MATQ_GEMV_T(4, 1) : MATQ_GEMV_T(2, 1);
+    else st = (r == 8) ? MATQ_GEMV_T(8, 2) : (r == 4) ? MATQ_GEMV_T(4, 2) : MATQ_GEMV_T(2, 2);
+#undef MATQ_GEMV_T
+    if (st != MATQ_OK) return st;
     return launch_status();
 }
