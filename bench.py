@@ -233,7 +233,8 @@ class DeviceStack:
                 for i in range(n):
                     K = S[i][4]
                     mq.gemv(planes[i], K, r, self.alpha[i], self.zero[i], self.x8[i][:B], y=self.y[nm][i],
-                            ovf_row_ptr=self.rp[i] if ep else None, ovf_col=self.col[i] if ep else None)
+                            ovf_row_ptr=self.rp[i] if ep else None, ovf_col=self.col[i] if ep else None,
+                            flags=mq.GEMV_AUTO | mq.GEMV_PDL)
             return run
 
         def gemm():

@@ -33,11 +33,29 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
         return launch_status();
     }
+    // Warp tile: 16*MT rows x K/SK.  Use two m-tiles per warp when there are plenty of rows (the staged activations
+    // are reused twice), then split K over as many warps as it takes to put about 16 warps on every SM.
+    const int sms = sm_count();
+    const int mt = (N >= (int64_t)32 * 2 * sms) ? 2 : 1;
+    const int64_t tiles = (N + 16 * mt - 1) / (16 * mt);
+    const int64_t n_qc = (K * r / 8 + 63) / 64;
+    int sk = 1;
+    while (sk < 8 && tiles * sk < (int64_t)16 * sms && n_qc / (2 * sk) >= 2) sk *= 2;
     int st;
-#define MATQ_GEMV_T(RR, NT) launch_gemv_tensor<RR, 2, NT, 4, 2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
-    if (B <= 8) st = (r == 8) ? MATQ_GEMV_T(8, 1) : (r == 4) ? MATQ_GEMV_T(4, 1) : MATQ_GEMV_T(2, 1);
-    else st = (r == 8) ? MATQ_GEMV_T(8, 2) : (r == 4) ? MATQ_GEMV_T(4, 2) : MATQ_GEMV_T(2, 2);
+#define MATQ_GEMV_T(RR, MT, NT, SK) launch_gemv_tensor<RR, MT, NT, SK>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+#define MATQ_GEMV_S(RR, MT, NT) ((sk == 8) ? MATQ_GEMV_T(RR, MT, NT, 8) : (sk == 4) ? MATQ_GEMV_T(RR, MT, NT, 4) : (sk == 2) ? MATQ_GEMV_T(RR, MT, NT, 2) : MATQ_GEMV_T(RR, MT, NT, 1))
+#define MATQ_GEMV_R(MT, NT) ((r == 8) ? MATQ_GEMV_S(8, MT, NT) : (r == 4) ? MATQ_GEMV_S(4, MT, NT) : MATQ_GEMV_S(2, MT, NT))
+    if (B <= 8) st = (mt == 2) ? MATQ_GEMV_R(2, 1) : MATQ_GEMV_R(1, 1);
+    else st = (mt == 2) ? MATQ_GEMV_R(2, 2) : MATQ_GEMV_R(1, 2);
+#undef MATQ_GEMV_R
+#undef MATQ_GEMV_S
 #undef MATQ_GEMV_T
+    if (st == MATQ_ERR_SHAPE) {   // the staged activations of this call do not fit in shared memory: FMA path
+        if (r == 8) launch_gemv_cuda_core<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        else if (r == 4) launch_gemv_cuda_core<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        return launch_status();
+    }
     if (st != MATQ_OK) return st;
     return launch_status();
 }
