@@ -59,7 +59,8 @@ enum matq_src_kind {
 enum matq_gemv_flags {
     MATQ_GEMV_AUTO = 0,        /* library picks the kernel */
     MATQ_GEMV_CUDA_CORE = 1,   /* fp32 FMA path */
-    MATQ_GEMV_TENSOR = 2,      /* warp-level tensor-core path (bf16 x bf16 -> fp32) */
+    MATQ_GEMV_TENSOR = 2,      /* warp-level tensor-core path (mma.sync, bf16 x bf16 -> fp32) */
+    MATQ_GEMV_TCGEN05 = 3,     /* tcgen05.mma path: unpacked weights as the TMEM A operand */
     MATQ_GEMV_PATH_MASK = 0xff,
     MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
                                   fetching weights while the previous kernel in the stream drains and

@@ -2,6 +2,7 @@
 #include "common.cuh"
 #include "gemv_cuda_core.cuh"
 #include "gemv_tensor.cuh"
+#include "gemv_tcgen05.cuh"
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
     (void)N; (void)K; (void)r; (void)B;
@@ -15,7 +16,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
                          void* workspace, size_t workspace_bytes, unsigned flags,
                          int32_t* dev_status, void* stream) {
     using namespace matq;
-    (void)workspace; (void)workspace_bytes; (void)dev_status;
+    (void)workspace; (void)workspace_bytes;
     if (N < 0 || K <= 0 || B < 1 || B > 16 || !x || (N > 0 && (!packed || !alpha || !zero || !y))) return MATQ_ERR_INVALID_ARG;
     if ((ovf_row_ptr == nullptr) != (ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits || !(r == 8 || r == 4 || r == 2)) return MATQ_ERR_UNSUPPORTED;
@@ -23,7 +24,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     if (ovf_row_ptr && K > 65536) return MATQ_ERR_SHAPE;
     if ((N > 0 && !aligned16(packed)) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
     const unsigned path = flags & MATQ_GEMV_PATH_MASK;
-    if (path > MATQ_GEMV_TENSOR || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
+    if (path > MATQ_GEMV_TCGEN05 || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
@@ -32,6 +33,13 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else if (r == 4) launch_gemv_cuda_core<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
         else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
         return launch_status();
+    }
+    if (path == MATQ_GEMV_AUTO || path == MATQ_GEMV_TCGEN05) {
+        int st5;
+        if (r == 8) st5 = t5::launch<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
+        else if (r == 4) st5 = t5::launch<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
+        else st5 = t5::launch<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
+        if (st5 != MATQ_ERR_SHAPE) return st5;     // a K too long for one cluster's shared memory falls through
     }
     // Warp tile: 16*MT rows x K/SK.  Use two m-tiles per warp when there are plenty of rows (the staged activations
     // are reused twice), then split K over as many warps as it takes to put about 16 warps on every SM.

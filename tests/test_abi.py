@@ -66,7 +66,7 @@ def test_argument_errors_are_found_on_the_host():
     assert gemv(r=3) == mq.ERR_UNSUPPORTED and gemv(c=4) == mq.ERR_UNSUPPORTED
     assert gemv(K=100, ldx=104) == mq.ERR_SHAPE and gemv(ldx=64) == mq.ERR_SHAPE and gemv(ldy=4) == mq.ERR_SHAPE
     assert gemv(packed=C.c_void_p(0x1004)) == mq.ERR_ALIGNMENT
-    assert gemv(flags=7) == mq.ERR_INVALID_ARG
+    assert gemv(flags=7) == mq.ERR_INVALID_ARG and gemv(flags=0x200) == mq.ERR_INVALID_ARG
     assert gemv(N=0) == mq.OK                                         # empty problem: nothing to launch
 
 

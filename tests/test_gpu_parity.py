@@ -164,7 +164,18 @@ def test_gemv_tensor_within_tolerance(r, N, K, B):
     assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
 
 
-@pytest.mark.parametrize("flags,tol", [(mq.GEMV_CUDA_CORE, TOL_FMA), (mq.GEMV_TENSOR, TOL_TENSOR), (mq.GEMV_AUTO, TOL_TENSOR)])
+@pytest.mark.parametrize("r", [8, 4, 2])
+@pytest.mark.parametrize("N,K,B", [(1024, 1024, 1), (300, 2304, 1), (130, 9216, 8), (77, 3584, 4), (3, 128, 16),
+                                   (257, 14336, 3), (64, 256, 5), (2304, 9216, 8), (500, 2432, 11), (129, 384, 2),
+                                   (9216, 2304, 1), (128, 128, 1)])
+def test_gemv_tcgen05_within_tolerance(r, N, K, B):
+    # default path: tcgen05.mma with the unpacked weights as the TMEM A operand
+    y, y_ref = _gemv_case(N, K, B, r, 500 + N + r, flags=mq.GEMV_TCGEN05)
+    assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
+
+
+@pytest.mark.parametrize("flags,tol", [(mq.GEMV_CUDA_CORE, TOL_FMA), (mq.GEMV_TENSOR, TOL_TENSOR), (mq.GEMV_TCGEN05, TOL_TENSOR),
+                                       (mq.GEMV_AUTO, TOL_TENSOR)])
 @pytest.mark.parametrize("r", [4, 2])
 @pytest.mark.parametrize("B", [1, 8])
 def test_gemv_extra_precision(r, B, flags, tol):
@@ -172,7 +183,7 @@ def test_gemv_extra_precision(r, B, flags, tol):
     assert np.abs(y - y_ref).max() <= tol * rms(y_ref)
 
 
-@pytest.mark.parametrize("flags", [mq.GEMV_CUDA_CORE, mq.GEMV_TENSOR])
+@pytest.mark.parametrize("flags", [mq.GEMV_CUDA_CORE, mq.GEMV_TENSOR, mq.GEMV_TCGEN05])
 @pytest.mark.parametrize("r", [8, 4, 2])
 def test_gemv_exact_integer_case(r, flags):
     # alpha = 1, z = 0, integer x: every partial sum is an exact fp32 integer, so the result must be exact.
