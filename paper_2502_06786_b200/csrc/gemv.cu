@@ -34,7 +34,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else launch_gemv_cuda_core<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
         return launch_status();
     }
-    if (path == MATQ_GEMV_AUTO || path == MATQ_GEMV_TCGEN05) {
+    if (path == MATQ_GEMV_TCGEN05) {   // opt-in: correct, but its per-CTA set-up still costs more than it saves at decode sizes
         int st5;
         if (r == 8) st5 = t5::launch<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         else if (r == 4) st5 = t5::launch<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
