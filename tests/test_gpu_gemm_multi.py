@@ -1,0 +1,122 @@
+"""GPU parity of the multi-precision dense forward (Eq. 7's F(S(Q(W, c), r), x) for every r in R) against the oracle.
+
+Tolerance: max|dY| <= 1e-2 * rms(Y_oracle) per output (tensor-core path); alpha / zero produced by the fused
+MinMax quantisation must equal the oracle's as fp32 values; the all-integer case must be exact.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2502_06786_b200 import binding as mq
+from paper_2502_06786_b200 import synth
+from tests.util import bf16_dev, dev, host, rms, status_word
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def _check(Ys, Yr, tol=TOL):
+    for yg, yr in zip(Ys, Yr):
+        err = np.abs(host(yg) - yr).max()
+        assert err <= tol * rms(yr), (err, rms(yr))
+
+
+@pytest.mark.parametrize("M,N,K", [(200, 264, 256), (128, 128, 64), (1, 8, 64), (384, 512, 1024), (130, 1000, 192)])
+def test_codes_source_all_precisions(M, N, K):
+    W = synth.normal_bf16((N, K), 0.02, 40 + M)
+    st, q, a, z = ref.quantize(W)
+    X = synth.normal_bf16((M, K), 1.0, 41 + M)
+    status = status_word()
+    Ys, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(8, 4, 2), alpha=dev(a), zero=dev(z), dev_status=status)
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, q, K, X, alpha=a, zero=z)
+    assert st == ref.OK
+    _check(Ys, Yr)
+    assert int(host(status)[0]) == mq.OK
+
+
+def test_bf16_source_quantizes_on_the_fly():
+    M, N, K = 160, 392, 512
+    W = synth.student_t_bf16((N, K), 3.0, 0.02, 50)
+    X = synth.normal_bf16((M, K), 1.0, 51)
+    Ys, a, z = mq.gemm_multi(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X))
+    st, Yr, ar, zr = ref.gemm_multi(ref.SRC_BF16, W, K, X)
+    assert np.array_equal(host(a), ar) and np.array_equal(host(z), zr)
+    _check(Ys, Yr)
+    # interpolated precisions (r = 6, 3) and a single output
+    Ys, _, _ = mq.gemm_multi(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), rs=(6, 3))
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_BF16, W, K, X, rs=(6, 3))
+    _check(Ys, Yr)
+
+
+@pytest.mark.parametrize("r,ep", [(4, False), (2, False), (2, True), (4, True), (8, False)])
+def test_packed_source(r, ep):
+    M, N, K = 96, 136, 256
+    q = synth.skewed_codes((N, K), 0.05, 224, 60 + r)
+    a = (np.abs(synth.bf16_bits_to_f32(synth.normal_bf16((N,), 0.01, 61))) + 1e-3).astype(np.float32)
+    z = synth.bf16_bits_to_f32(synth.normal_bf16((N,), 40.0, 62)).astype(np.float32) + 128
+    X = synth.normal_bf16((M, K), 1.0, 63)
+    sp = ref.slice_pack(q, r, extra_precision=ep)
+    rp, col = (sp["ovf_row_ptr"], sp["ovf_col"]) if (ep and r < 8) else (None, None)
+    Ys, _, _ = mq.gemm_multi(mq.SRC_PACKED, dev(sp["packed"]), K, bf16_dev(X), rs=(r,), alpha=dev(a), zero=dev(z),
+                             extra_precision=ep, ovf_row_ptr=dev(rp) if rp is not None else None,
+                             ovf_col=dev(col if col.size else np.zeros(1, np.uint16)) if rp is not None else None)
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_PACKED, sp["packed"], K, X, rs=(r,), alpha=a, zero=z, extra_precision=ep,
+                                  ovf_row_ptr=rp, ovf_col=col)
+    assert st == ref.OK
+    _check(Ys, Yr)
+    # the same result from the codes with Eq. 8 applied on the fly
+    Yc, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(r,), alpha=dev(a), zero=dev(z), extra_precision=ep)
+    assert torch.equal(Yc[0], Ys[0])
+
+
+def test_exact_integer_case_and_independence_of_outputs():
+    # alpha = 1, z = 0, integer activations: every partial sum is an exact fp32 integer
+    M, N, K = 128, 128, 512
+    q = synth.uniform_codes((N, K), 70)
+    X = synth.small_int_bf16((M, K), -4, 4, 71)
+    a = np.ones(N, np.float32); z = np.zeros(N, np.float32)
+    Ys, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), alpha=dev(a), zero=dev(z))
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, q, K, X, alpha=a, zero=z)
+    for yg, yr in zip(Ys, Yr):
+        assert np.array_equal(host(yg).astype(np.float64), yr)
+    # each precision alone gives the same bits as in the fused call
+    for i, r in enumerate((8, 4, 2)):
+        Y1, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(r,), alpha=dev(a), zero=dev(z))
+        assert torch.equal(Y1[0], Ys[i])
+
+
+def test_matches_decode_gemv_and_full_path():
+    # quantize -> slice_pack -> gemv on M rows one batch at a time == the dense forward
+    M, N, K = 8, 256, 512
+    W = synth.normal_bf16((N, K), 0.02, 80)
+    X = synth.normal_bf16((M, K), 1.0, 81)
+    Ys, a, z = mq.gemm_multi(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X))
+    q, a2, z2 = mq.quantize(bf16_dev(W))
+    assert torch.equal(a, a2) and torch.equal(z, z2)
+    for i, r in enumerate((8, 4, 2)):
+        sp = mq.slice_pack(q, r)
+        y = mq.gemv(sp["packed"], K, r, a, z, bf16_dev(X))
+        assert np.abs(host(y) - host(Ys[i])).max() <= 1e-3 * rms(host(y))
+
+
+def test_argument_errors_and_empty():
+    lib = mq._lib
+    fake = C.c_void_p(0x1000)
+    rs3 = (C.c_int * 3)(8, 4, 2)
+    ys = (C.c_void_p * 3)(0x1000, 0x1000, 0x1000)
+
+    def call(src=mq.SRC_CODES8, N=128, K=128, c=8, M=128, ldx=128, rs=rs3, n_r=3, ldy=128, ws=fake, wsb=1 << 30):
+        return lib.matq_gemm_multi(src, fake, N, K, c, fake, fake, 0, None, None, fake, M, ldx, rs, n_r, ys, ldy, ws, wsb, None, None)
+    assert call(n_r=4) == mq.ERR_INVALID_ARG and call(n_r=0) == mq.ERR_INVALID_ARG
+    assert call(src=7) == mq.ERR_INVALID_ARG
+    assert call(c=4) == mq.ERR_UNSUPPORTED
+    assert call(rs=(C.c_int * 3)(8, 8, 2)) == mq.ERR_INVALID_ARG          # precisions must be distinct
+    assert call(rs=(C.c_int * 3)(9, 4, 2)) == mq.ERR_UNSUPPORTED
+    assert call(K=100, ldx=104) == mq.ERR_SHAPE and call(N=132, ldy=132) == mq.ERR_SHAPE
+    assert call(src=mq.SRC_PACKED, n_r=3) == mq.ERR_INVALID_ARG            # one plane, one precision
+    assert call(wsb=16) == mq.ERR_WORKSPACE and call(ws=None) == mq.ERR_WORKSPACE
+    assert call(M=0) == mq.OK
+    assert mq.gemm_multi_workspace_bytes(mq.SRC_BF16, 128, 128, 128, 3) >= 128 * 128 * (1 + 6) + 512
