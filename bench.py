@@ -10,7 +10,10 @@ A step is one pass of the whole path over the Gemma-2-2B-shaped MLP stack
   decode GEMV  r=4  B=1, B=8            packed plane, bf16 x -> fp32 y
   decode GEMV  r=2  B=1, B=8
   decode GEMV  r=2  extra precision, B=1
-  multi-precision forward r={8,4,2}     M tokens, codes -> three fp32 outputs (when the library provides it)
+
+The dense multi-precision forward (Eq. 7) has no place in a decode-shaped workload (1 or 8 activations per layer);
+it is measured on its own configuration, the Mistral-7B-shaped co-training forward (W 14336x4096, 4096 tokens,
+r = 8, 4, 2 in one call), and reported in the same JSON line under `gemm_multi_cfg4` with its tensor roofline.
 
 Every matrix of the stack has its own buffers, so each stage streams far more
 than the L2 holds.  `value` is the algorithmic HBM bytes of the step divided by
@@ -42,7 +45,6 @@ from paper_2502_06786_b200 import synth  # noqa: E402
 
 METRIC = "sliced int{8,4,2} GEMV HBM GB/s (% of peak); multi-precision GEMM TFLOP/s"
 CONFIG_ID = 2
-GEMM_M = 128          # tokens of the multi-precision forward stage at this (decode-shaped) workload
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -175,11 +177,6 @@ class DeviceStack:
                   for nm, B in (("g4b1", 1), ("g4b8", 8), ("g2b1", 1), ("g2b8", 8), ("g2ep", 1))}
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.has_gemm = self._probe_gemm()
-        if self.has_gemm:
-            self.Xg = [torch.empty((GEMM_M, K), dtype=torch.bfloat16, device=dev) for (_, _, _, N, K) in shapes]
-            self.Yg = [[torch.empty((GEMM_M, N), dtype=f32, device=dev) for _ in range(3)] for (_, _, _, N, K) in shapes]
-            ws = max(mq.gemm_multi_workspace_bytes(mq.SRC_CODES8, GEMM_M, N, K, 3) for (_, _, _, N, K) in shapes)
-            self.ws = torch.empty(max(ws, 16), dtype=u8, device=dev)
         self.W_pinned = self.x_pinned = None
         self.upload(W_host, x_host)
 
@@ -202,9 +199,6 @@ class DeviceStack:
         for i, (W, x) in enumerate(zip(W_host, x_host)):
             self.W[i].view(torch.uint16).copy_(torch.from_numpy(W))
             self.x8[i].view(torch.uint16).copy_(torch.from_numpy(x))
-            if self.has_gemm:
-                reps = GEMM_M // 8
-                self.Xg[i].copy_(self.x8[i].repeat(reps, 1))
         torch.cuda.synchronize()
 
     # stage-major plan: name -> (callable over the whole stack, kernels launched, algorithmic bytes, flops)
@@ -237,12 +231,6 @@ class DeviceStack:
                             flags=mq.GEMV_AUTO | mq.GEMV_PDL)
             return run
 
-        def gemm():
-            for i in range(n):
-                K = S[i][4]
-                mq.gemm_multi(mq.SRC_CODES8, self.q[i], K, self.Xg[i], alpha=self.alpha[i], zero=self.zero[i],
-                              Ys=self.Yg[i], workspace=self.ws)
-
         nnz = getattr(self, "nnz", [0] * n)
         plan = [
             ("quantize", quant, n, sum(bytes_quantize(N, K) for (_, _, _, N, K) in S), 0),
@@ -255,10 +243,6 @@ class DeviceStack:
             ("gemv_r2_ep_b1", gemv("g2ep", 2, 1, True), n,
              sum(bytes_gemv(N, K, 2, 1, z) for (_, _, _, N, K), z in zip(S, nnz)), 0),
         ]
-        if self.has_gemm:
-            plan.append(("gemm_multi_r842", gemm, None,
-                         sum(N * K + 2 * GEMM_M * K + 3 * 4 * GEMM_M * N for (_, _, _, N, K) in S),
-                         sum(3 * 2 * GEMM_M * N * K for (_, _, _, N, K) in S)))
         return plan
 
 
@@ -361,6 +345,13 @@ def run_cuda(args, rank, world, local_rank):
     # ------------------------------------------------------------------ end to end from host buffers
     e2e = e2e_leg(st, plan, W_host, x_host, args, torch, world, dist if world > 1 else None)
 
+    cfg4 = None
+    if st.has_gemm and world == 1 and not args.no_cfg4:
+        for t in (st.W, st.q, st.p4, st.p2):       # free the stack's large buffers first
+            t.clear()
+        torch.cuda.empty_cache()
+        cfg4 = gemm_cfg4(mq, torch, peaks)
+
     out = None
     if rank == 0:
         out = {
@@ -370,17 +361,47 @@ def run_cuda(args, rank, world, local_rank):
             "config": {"workload": f"configs[1] Gemma-2-2B-shaped MLP decode stack, {args.layers} layers x (gate,up 9216x2304; down 2304x9216), "
                                    "bf16 N(0,0.02) weights, x bf16 N(0,1)",
                        "step": "quantize -> slice_pack r=4 -> slice_pack r=2 + extra-precision lists -> gemv r=4 B=1,8 -> gemv r=2 B=1,8 -> gemv r=2 E.P. B=1"
-                               + (f" -> gemm_multi r=8,4,2 M={GEMM_M}" if st.has_gemm else ""),
+                               + "; dense multi-precision forward measured separately (gemm_multi_cfg4)",
                        "value_definition": "algorithmic HBM bytes of the step / device time; one CUDA graph per stage",
                        "l2": "inputs larger than L2: every matrix has its own buffers, each stage streams >= 0.4 GB",
                        "parallelism": "one independent stack per GPU (rows are independent; no collective)" if world > 1 else "single GPU",
                        "overflow_fraction_r2": round(sum(st.nnz) / sum(N * K for (_, _, _, N, K) in shapes), 6)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "stages": stages, "roofline": roofline,
         }
+        if cfg4 is not None:
+            out["gemm_multi_cfg4"] = cfg4
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     return out, st
+
+
+def gemm_cfg4(mq, torch, peaks, reps=5):
+    """configs[3]: Mistral-7B-shaped co-training forward, one fused call: quantize + slice r = 8, 4, 2 + three GEMMs."""
+    N, K, M = 14336, 4096, 4096
+    W = torch.from_numpy(synth.normal_bf16((N, K), 0.02, synth.seed_for(4, 0))).cuda().view(torch.bfloat16)
+    X = torch.from_numpy(synth.normal_bf16((M, K), 1.0, synth.seed_for(4, 500))).cuda().view(torch.bfloat16)
+    Ys = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(3)]
+    a = torch.empty(N, dtype=torch.float32, device="cuda"); z = torch.empty_like(a)
+    ws = torch.empty(mq.gemm_multi_workspace_bytes(mq.SRC_BF16, M, N, K, 3), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        mq.gemm_multi(mq.SRC_BF16, W, K, X, alpha=a, zero=z, Ys=Ys, workspace=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        mq.gemm_multi(mq.SRC_BF16, W, K, X, alpha=a, zero=z, Ys=Ys, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    flops = 3 * 2.0 * M * N * K
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"workload": "configs[3] W 14336x4096 bf16, X 4096x4096 bf16, r = 8, 4, 2, fp32 outputs, one matq_gemm_multi(MATQ_SRC_BF16) call",
+            "ms": round(ms, 3), "TFLOPs": round(tf, 1), "frac_tensor_sustained": round(tf / peaks["bf16_tflops_sustained"], 4),
+            "frac_tensor_burst": round(tf / peaks["bf16_tflops"], 4), "flops": flops,
+            "roofline": {"kernel": "gemm_multi (quantize + expand + rowsum + tcgen05 GEMM)", "bound": "tensor", "achieved": round(tf, 1),
+                         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": round(tf / peaks["bf16_tflops_sustained"], 4),
+                         "traffic": None, "peak_source": peaks["source"] + " (sustained)"}}
 
 
 def e2e_leg(st, plan, W_host, x_host, args, torch, world, dist):
@@ -494,6 +515,7 @@ def main():
     ap.add_argument("--layers", type=int, default=synth.WORKLOADS[CONFIG_ID]["layers"])
     ap.add_argument("--cpu-sample-layers", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cfg4", action="store_true", help="skip the extra Mistral-7B-shaped gemm_multi measurement")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
