@@ -169,6 +169,29 @@ int matq_gemm_multi(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
                     void *workspace, size_t workspace_bytes,
                     int32_t *dev_status, void *stream);
 
+/*
+ * (5) matq_gemm_multi without a workspace argument.  The paper has no counterpart to this call: it exists for
+ *     callers that cannot obtain device memory when they call the library (a serving loop whose memory was divided
+ *     up at start-up and that must not call cudaMalloc on the request path, because that call synchronises the
+ *     device and can fail under fragmentation; a plug-in inside another framework's memory pool).  The scratch
+ *     that matq_gemm_multi takes from its workspace comes from an array built into the library's device image:
+ *     matq_gemm_multi_static_max_bytes() bytes (16 MiB) on every GPU that loads the library, held until exit.
+ *   Arguments and results are those of matq_gemm_multi.  Nothing is allocated or freed by this call.
+ *   MATQ_ERR_WORKSPACE is returned, before anything is launched, when
+ *     matq_gemm_multi_workspace_bytes(src_kind, M, N, K, n_r) > matq_gemm_multi_static_max_bytes().
+ *   The first call on each device looks up the array's device address (that device must be current) and should be
+ *   made before any stream capture begins.  All calls on a GPU share the array and it keeps the previous call's
+ *   contents; none of it needs to start at zero, but calls that overlap on the GPU race on it and must be ordered
+ *   by the caller (one stream, or events between streams).
+ */
+size_t matq_gemm_multi_static_max_bytes(void);
+int matq_gemm_multi_static(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
+                           float *alpha, float *zero, int extra_precision,
+                           const int32_t *ovf_row_ptr, const uint16_t *ovf_col,
+                           const void *X, int64_t M, int64_t ldx,
+                           const int *rs, int n_r, float *const *Y, int64_t ldy,
+                           int32_t *dev_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,8 @@ GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_PDL = 0, 1, 2, 3, 0x1
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize",
            "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv",
-           "matq_gemm_multi_workspace_bytes", "matq_gemm_multi"]
+           "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
+           "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
 
 
 class MatqError(RuntimeError):
@@ -57,6 +58,11 @@ def _load():
     lib.matq_gemm_multi.restype = i32
     lib.matq_gemm_multi.argtypes = [i32, vp, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, i64,
                                     C.POINTER(C.c_int), i32, C.POINTER(C.c_void_p), i64, vp, sz, vp, vp]
+    lib.matq_gemm_multi_static_max_bytes.restype = sz
+    lib.matq_gemm_multi_static_max_bytes.argtypes = []
+    lib.matq_gemm_multi_static.restype = i32
+    lib.matq_gemm_multi_static.argtypes = [i32, vp, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, i64,
+                                           C.POINTER(C.c_int), i32, C.POINTER(C.c_void_p), i64, vp, vp]
     return lib
 
 
@@ -212,3 +218,26 @@ def gemm_multi(src_kind, Wsrc, K, X, rs=(8, 4, 2), alpha=None, zero=None, extra_
                               workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream())
     _check(st, "matq_gemm_multi")
     return Ys, alpha, zero
+
+
+def gemm_multi_static_max_bytes() -> int:
+    return int(_lib.matq_gemm_multi_static_max_bytes())
+
+
+def gemm_multi_static(src_kind, Wsrc, K, X, Ys, alpha, zero, rs=(8, 4, 2), extra_precision=False,
+                      ovf_row_ptr=None, ovf_col=None, dev_status=None, c=8, raise_on_error=True):
+    """matq_gemm_multi_static: the dense forward with the library's built-in scratch.
+
+    For callers that cannot allocate device memory at call time.  Unlike ``gemm_multi`` this wrapper allocates
+    nothing either: the outputs ``Ys`` (one fp32 [M, N] tensor per precision), ``alpha`` and ``zero`` must be passed in.
+    Returns the status (raises ``MatqError`` unless ``raise_on_error`` is false).
+    """
+    _dev(X, torch.bfloat16, "X", 2)
+    _dev(Wsrc, torch.bfloat16 if src_kind == SRC_BF16 else torch.uint8, "Wsrc", 2)
+    N, M = Wsrc.shape[0], X.shape[0]
+    rs_arr = (C.c_int * len(rs))(*rs)
+    y_arr = (C.c_void_p * len(rs))(*[y.data_ptr() for y in Ys])
+    st = _lib.matq_gemm_multi_static(src_kind, _ptr(Wsrc), N, K, c, _ptr(alpha), _ptr(zero), int(bool(extra_precision)),
+                                     _ptr(ovf_row_ptr), _ptr(ovf_col), _ptr(X), M, _ld(X, K), rs_arr, len(rs),
+                                     y_arr, _ld(Ys[0], N), _ptr(dev_status), _stream())
+    return _check(st, "matq_gemm_multi_static", raise_on_error)

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmatq.so")
-SOURCES = ["api.cu", "quantize.cu", "slice_pack.cu", "gemv.cu", "gemm_multi.cu"]
+SOURCES = ["api.cu", "quantize.cu", "slice_pack.cu", "gemv.cu", "gemm_multi.cu", "gemm_multi_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-Wno-deprecated-gpu-targets"]
 
