@@ -3,4 +3,4 @@
 ``binding`` wraps the C ABI of ``libmatq.so`` (declared in ``include/matq.h``);
 ``synth`` holds the seeded synthetic inputs; ``build`` compiles the library.
 """
-__all__ = ["binding", "synth", "build"]
+__all__ = ["binding", "synth", "build", "shard"]
