@@ -1,4 +1,4 @@
-// Decode GEMV on the fifth-generation tensor cores (tcgen05.mma, accumulators and the A operand in tensor memory).
+// Decode GEMV on the fifth-generation tensor cores (tcgen05.mma, accumulator and the A operand in tensor memory).
 //
 // Why not the warp-level MMA: on B200 one mma.sync.m16n8k16 occupies a sub-partition's legacy tensor pipe for
 // about 32 cycles, so a decode GEMV (one batch column = 7/8 padding per MMA) is bound by that pipe well below the
@@ -19,18 +19,23 @@
 // word, and x' is staged in that same order.  The constant 128 contributes 128 * sum(x') to every row; it is removed
 // in the epilogue with the separately accumulated sum.
 //
-// Data movement.  Every thread of the first four warps issues one bulk asynchronous copy (cp.async.bulk) for its
-// row's slice of the packed plane, completion counted on one mbarrier per 32 rows; all of a CTA's bytes are in flight
-// at once and are requested BEFORE the kernel waits for its predecessor in the stream (programmatic dependent
-// launch), so a layer's weights stream in while the previous layer still computes.  TMEM is allocated before the
-// dependents are released, so a waiting successor can never starve a predecessor of tensor memory.
+// Warp roles (13 warps):
+//   warps 0-7   two "unpack" warpgroups.  Each owns three TMEM slots of 32 columns (4 instructions' worth of A) and
+//               fills them round-robin from the shared-memory weight tile; an mbarrier per slot says "ready", the
+//               tcgen05.commit of the instructions that read a slot says "free".  They start as soon as the weights
+//               land, i.e. BEFORE the kernel's predecessor in the stream has finished.
+//   warps 8-11  wait for the predecessor (programmatic dependent launch), stage x' and the two sums, signal "x ready".
+//   warp 12     one lane issues the TMA copies of the weight tile (before the dependency wait) and later all MMAs,
+//               always in slot order, so the single accumulator is summed in a fixed order (deterministic results).
 //
-// Four warpgroups take the 16-byte chunks of the slice round-robin, each with two TMEM slots (tcgen05.commit frees a
-// slot when the MMAs that read it retire) and its own accumulator; the four accumulators are added in a fixed order.
-// Slices of K (grid.y > 1) form a thread-block cluster and are summed through distributed shared memory in rank
-// order.  No global scratch, no atomics: results are deterministic.
+// Data movement.  The CTA's slice of the packed plane is fetched as 128-byte x 128-row boxes of a 2-D tensor map over
+// the plane (uint8, 128-byte swizzle so that 32 rows can be read 16 bytes at a time without bank conflicts; rows and
+// bytes outside the matrix arrive as zeros).  No multicast.  TMEM is allocated before the dependents are released, so
+// a waiting successor can never starve a predecessor of tensor memory.  Slices of K (grid.y > 1) form a thread-block
+// cluster and are summed through distributed shared memory in rank order.  No global scratch, no atomics.
 #pragma once
 #include <cooperative_groups.h>
+#include <cuda.h>
 
 #include "common.cuh"
 
@@ -38,18 +43,19 @@ namespace matq {
 namespace t5 {
 namespace cg = cooperative_groups;
 
-constexpr int kThreads = 512;
-constexpr int kWarpgroups = 4;
+constexpr int kUnpackWarps = 8, kStageWarps = 4;
+constexpr int kThreads = 32 * (kUnpackWarps + kStageWarps + 1);
 constexpr int kRows = 128;                   // M of the MMA = TMEM lanes
 constexpr int kNB = 16;                      // N of the MMA = batch columns (padded)
-constexpr int kStepBytes = 512;              // x' bytes of one K = 16 instruction: [k-half][n-group][8 n][8 k] bf16
-constexpr int kSlotCols = 16;                // TMEM columns of one A slot = two K = 16 instructions
-constexpr int kTmemCols = 256;               // 4 accumulators x 16 + 4 warpgroups x 2 slots x 16 = 192 -> 256
-constexpr int kAccCol = 0, kSlotCol = 64;
+constexpr int kSlotCols = 32;                // TMEM columns of one A slot = four K = 16 instructions
+constexpr int kSlots = 3;                    // slots per unpack warpgroup
+constexpr int kTmemCols = 256;               // accumulator 16 + 2 warpgroups x 3 slots x 32 = 208 -> 256
+constexpr int kAccCol = 0, kSlotCol = 32;
+constexpr int kBoxBytes = 128 * kRows;       // one TMA box: 128 bytes of 128 rows
+constexpr int kMaxBoxes = 8;
 constexpr uint32_t kSpinLimit = 1u << 22;    // mbarrier polls before a wait gives up
 
 struct Params {
-    const uint8_t* packed;
     const float* alpha;
     const float* zero;
     const int32_t* ovf_row_ptr;
@@ -60,8 +66,8 @@ struct Params {
     int64_t N, K, ldx, ldy;
     int64_t row_bytes;
     int B;
-    int slice_bytes;     // bytes of a row handled by one CTA (multiple of 16; the last slice may be shorter)
-    int tile_stride;     // bytes between rows of the shared-memory weight tile (16 mod 128)
+    int slice_bytes;     // bytes of a row handled by one CTA (multiple of 128 except possibly the last slice)
+    int step_bytes;      // x' bytes of one instruction: 256 (B <= 8: both column groups read the same 128 bytes) or 512
     int pdl;
 };
 
@@ -99,14 +105,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     return done != 0;
 }
-
-// Shared-memory matrix descriptor of one x' step: K-major, no swizzle, 8 x 16-byte core matrices; the two k-halves
-// are 256 bytes apart (leading byte offset), the two groups of 8 batch columns 128 bytes (stride byte offset).
-__device__ __forceinline__ uint64_t b_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)(256 >> 4) << 16) | ((uint64_t)(128 >> 4) << 32) | (1ull << 46);
-}
-// kind::f16, D = fp32, A = B = bf16, both K-major, N = 16, M = 128
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kNB >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
 // Steps (K = 16 instructions) per 16-byte chunk of a row, and activations covered by one step.
 template <int R> struct Fmt;
@@ -152,51 +150,59 @@ __device__ __forceinline__ void stage_step(const __nv_bfloat16* xk, uint4& h0, u
     }
 }
 
-template <int R>
-__global__ void __launch_bounds__(kThreads, 1)
-gemv_tcgen05(const Params P) {
-    constexpr int sh = kCodeBits - R;
-    constexpr int kStepsPerChunk = Fmt<R>::kStepsPerChunk;
-    constexpr int kKPerStep = Fmt<R>::kKPerStep;
-    constexpr int kSlotBytes = 16 * 2 / kStepsPerChunk;       // row bytes unpacked into one slot (two steps)
-    constexpr int kWordsPerSlot = kSlotBytes / 4;
+// Shared-memory matrix descriptor of one x' step: K-major, no swizzle, 8 x 16-byte core matrices.  The two k-halves
+// are lbo bytes apart (leading byte offset), the two groups of 8 batch columns sbo bytes (stride byte offset; 0 makes
+// columns 8..15 re-read columns 0..7, whose results are never used when B <= 8).
+__device__ __forceinline__ uint64_t b_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+// kind::f16, D = fp32, A = B = bf16, both K-major, N = 16, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kNB >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t s_wbar[4];                 // weight rows of TMEM lane quadrant q have landed
-    __shared__ __align__(8) uint64_t s_free[kWarpgroups][2];    // A slot may be overwritten
-    __shared__ __align__(8) uint64_t s_done[kWarpgroups];       // accumulator of the warpgroup is final
+template <int R>
+__global__ void __launch_bounds__(kThreads, 2)
+gemv_tcgen05(const __grid_constant__ CUtensorMap tm_w, const Params P) {
+    constexpr int sh = kCodeBits - R;
+    constexpr int kKPerStep = Fmt<R>::kKPerStep;
+    constexpr int kSlotBytes = 16 * 4 / Fmt<R>::kStepsPerChunk;   // row bytes unpacked into one slot (four steps): 32 or 16
+    constexpr int kWordsPerSlot = kSlotBytes / 4;
+    constexpr int kPairsPerWord = kSlotCols / kWordsPerSlot;
+
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t s_wbar[kMaxBoxes];          // box b of the weight tile has landed
+    __shared__ __align__(8) uint64_t s_ready[2][kSlots];         // slot filled by all 128 threads of its warpgroup
+    __shared__ __align__(8) uint64_t s_free[2][kSlots];          // the instructions that read the slot have retired
+    __shared__ __align__(8) uint64_t s_xready, s_done;
     __shared__ uint32_t s_tmem;
-    __shared__ float s_red[2][kThreads / 32][kNB];
+    __shared__ float s_red[2][kStageWarps][kNB];
     __shared__ float s_sumx[kNB], s_sumxp[kNB];
     __shared__ float s_part[kRows][kNB];                         // this CTA's partial outputs (cluster reduction)
+    __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wg = warp >> 2, quad = warp & 3;                  // warp may touch TMEM lanes [32*quad, 32*quad + 32)
-    const int row_l = quad * 32 + lane;                         // the row this thread unpacks and finishes
     const int split = blockIdx.y, n_split = gridDim.y;
     const int64_t row0 = (int64_t)blockIdx.x * kRows;
     const int64_t slice_off = (int64_t)split * P.slice_bytes;
     const int my_bytes = (int)min((int64_t)P.slice_bytes, P.row_bytes - slice_off);    // multiple of 16, >= 16
-    const int n_chunks = my_bytes / kSlotBytes;                 // slots to fill in this CTA
-    const int n_steps = n_chunks * 2;
-    const int rows_here = (int)min((int64_t)kRows, P.N - row0);
+    const int n_boxes = (my_bytes + 127) / 128;
+    const int n_slots = (my_bytes + kSlotBytes - 1) / kSlotBytes;
+    const int n_steps = n_slots * 4;
 
-    unsigned char* wt = smem_raw;                               // [128][tile_stride]
-    unsigned char* xs = smem_raw + (size_t)kRows * P.tile_stride;   // [steps][512]
+    unsigned char* wt = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);      // [box][128 rows][128 B], swizzled
+    unsigned char* xs = wt + (size_t)n_boxes * kBoxBytes;                              // [step][step_bytes]
 
     // ---- barriers, tensor memory, weight copies: nothing here depends on the previous kernel
     if (tid == 0) {
-        for (int q = 0; q < 4; ++q) {
-            const int rq = max(0, min(32, rows_here - q * 32));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_wbar[q])));
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&s_wbar[q])), "r"(rq * my_bytes) : "memory");
-        }
-        for (int w = 0; w < kWarpgroups; ++w) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_free[w][0])));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_free[w][1])));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_done[w])));
-        }
+        for (int b = 0; b < kMaxBoxes; ++b) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_wbar[b])));
+        for (int w = 0; w < 2; ++w)
+            for (int sl = 0; sl < kSlots; ++sl) {
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 128;" ::"r"(smem_u32(&s_ready[w][sl])));
+                asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_free[w][sl])));
+            }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&s_xready)), "r"(32 * kStageWarps));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_done)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_timeout = 0;
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kTmemCols) : "memory");
@@ -206,148 +212,139 @@ gemv_tcgen05(const Params P) {
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s_tmem;
+    if (P.pdl) asm volatile("griddepcontrol.launch_dependents;");
 
-    if (tid < rows_here) {
-        const uint8_t* src = P.packed + (row0 + tid) * P.row_bytes + slice_off;
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_u32(wt + (size_t)tid * P.tile_stride)), "l"(src), "r"(my_bytes), "r"(smem_u32(&s_wbar[tid >> 5])) : "memory");
-    }
-    float a_pre = 0.f, z_pre = 0.f;
-    if (wg == 0 && row0 + row_l < P.N) {
-        a_pre = P.alpha[row0 + row_l];
-        z_pre = P.zero[row0 + row_l];
-    }
-
-    if (P.pdl) {
-        asm volatile("griddepcontrol.launch_dependents;");
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-    }
-
-    // ---- activations: zero the x' tile, then write the rows of the batch columns in use; sums on the way
-    {
-        uint4* xz = reinterpret_cast<uint4*>(xs);
-        for (int i = tid; i < n_steps * (kStepBytes / 16); i += kThreads) xz[i] = make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
-    {
-        // item = (step, batch column); 512 threads cover 32 steps x 16 columns per pass, a thread keeps its column
-        const int bcol = tid & (kNB - 1);
-        const int64_t k_base = slice_off * 8 / R;               // first activation of the slice
-        float sx = 0.f, sxp = 0.f;
-        if (bcol < P.B) {
-            for (int st = tid >> 4; st < n_steps; st += kThreads / kNB) {
-                const int64_t k = k_base + (int64_t)st * kKPerStep;
-                if (k < P.K) {
-                    uint4 h0, h1;
-                    stage_step<R>(P.x + (int64_t)bcol * P.ldx + k, h0, h1, sx, sxp);
-                    unsigned char* base = xs + (size_t)st * kStepBytes + (bcol >> 3) * 128 + (bcol & 7) * 16;
-                    *reinterpret_cast<uint4*>(base) = h0;
-                    *reinterpret_cast<uint4*>(base + 256) = h1;
-                }
+    if (warp < kUnpackWarps) {
+        // ================= unpack warpgroups: weights -> bf16x2 -> TMEM slots; warpgroup 0 also finishes the rows
+        const int wg = warp >> 2, quad = warp & 3;
+        const int row_l = quad * 32 + lane;
+        bool ok = true;
+        float a_pre = 0.f, z_pre = 0.f;
+        if (wg == 0 && row0 + row_l < P.N) { a_pre = P.alpha[row0 + row_l]; z_pre = P.zero[row0 + row_l]; }
+        int landed = 0;                                          // boxes this thread has already waited for
+        int it = 0;
+        for (int s = wg; s < n_slots; s += 2, ++it) {
+            const int slot = it % kSlots;
+            if (it >= kSlots) ok &= mbar_wait(smem_u32(&s_free[wg][slot]), (uint32_t)(it / kSlots - 1) & 1u);
+            const int off = s * kSlotBytes;
+            const int box = off >> 7;
+            while (landed <= box) { ok &= mbar_wait(smem_u32(&s_wbar[landed]), 0); ++landed; }
+            const unsigned char* rowp = wt + (size_t)box * kBoxBytes + row_l * 128;
+            const int j0 = (off & 127) >> 4;
+            uint32_t wv[8];
+            {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + ((j0 ^ (row_l & 7)) << 4));
+                wv[0] = v.x; wv[1] = v.y; wv[2] = v.z; wv[3] = v.w;
             }
-        }
-        // lanes l and l + 16 hold the same column: fold, then one value per (warp, column)
-        sx += __shfl_xor_sync(0xffffffffu, sx, 16);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 16);
-        if (lane < kNB) { s_red[0][warp][lane] = sx; s_red[1][warp][lane] = sxp; }
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // x' was written with ordinary stores, the MMA reads it
-    __syncthreads();
-    if (tid < kNB) {
-        float sx = 0.f, sxp = 0.f;
-        for (int w = 0; w < kThreads / 32; ++w) { sx += s_red[0][w][tid]; sxp += s_red[1][w][tid]; }
-        s_sumx[tid] = sx;
-        s_sumxp[tid] = sxp;
-    }
-
-    // ---- main loop: warpgroup wg fills slots with chunks wg, wg + 4, ...; one thread issues the MMAs
-    bool ok = mbar_wait(smem_u32(&s_wbar[quad]), 0);
-    const unsigned char* my_row = wt + (size_t)row_l * P.tile_stride;
-    const uint32_t acc_addr = tmem + kAccCol + wg * kNB;
-    int it = 0;
-    for (int c = wg; c < n_chunks; c += kWarpgroups, ++it) {
-        const int slot = it & 1;
-        if (it >= 2) ok &= mbar_wait(smem_u32(&s_free[wg][slot]), ((it >> 1) - 1) & 1);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t wv[4];
-        if (kWordsPerSlot == 4) {
-            const uint4 v = *reinterpret_cast<const uint4*>(my_row + (size_t)c * 16);
-            wv[0] = v.x; wv[1] = v.y; wv[2] = v.z; wv[3] = v.w;
-        } else {
-            const uint2 v = *reinterpret_cast<const uint2*>(my_row + (size_t)c * 8);
-            wv[0] = v.x; wv[1] = v.y; wv[2] = 0; wv[3] = 0;
-        }
-        uint32_t a[kSlotCols];
+            if (kWordsPerSlot == 8) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + (((j0 + 1) ^ (row_l & 7)) << 4));
+                wv[4] = v.x; wv[5] = v.y; wv[6] = v.z; wv[7] = v.w;
+            }
+            uint32_t a[kSlotCols];
 #pragma unroll
-        for (int i = 0; i < kSlotCols; ++i) {
-            constexpr int kPairsPerWord = kSlotCols / kWordsPerSlot;
-            a[i] = field_pair<R>(wv[i / kPairsPerWord], i % kPairsPerWord);
-        }
-        const uint32_t slot_addr = tmem + ((uint32_t)(quad * 32) << 16) + kSlotCol + (wg * 2 + slot) * kSlotCols;
-        asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-                     ::"r"(slot_addr), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]),
-                       "r"(a[8]), "r"(a[9]), "r"(a[10]), "r"(a[11]), "r"(a[12]), "r"(a[13]), "r"(a[14]), "r"(a[15]) : "memory");
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
-        if ((tid & 127) == 0) {
+            for (int i = 0; i < kSlotCols; ++i) a[i] = field_pair<R>(wv[i / kPairsPerWord], i % kPairsPerWord);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_addr = tmem + kSlotCol + (wg * 2 + slot) * kSlotCols;
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                const uint64_t bd = b_desc(smem_u32(xs + (size_t)(2 * c + s) * kStepBytes));
-                const uint32_t accumulate = (it > 0 || s > 0) ? 1u : 0u;
-                asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p; }"
-                             ::"r"(acc_addr), "r"(a_addr + s * 8), "l"(bd), "r"(kIdesc), "r"(accumulate) : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_free[wg][slot])) : "memory");
-            if (c + kWarpgroups >= n_chunks)
-                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_done[wg])) : "memory");
+            const uint32_t slot_addr = tmem + ((uint32_t)(quad * 32) << 16) + kSlotCol + (wg * kSlots + slot) * kSlotCols;
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                         "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                         ::"r"(slot_addr), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]),
+                           "r"(a[8]), "r"(a[9]), "r"(a[10]), "r"(a[11]), "r"(a[12]), "r"(a[13]), "r"(a[14]), "r"(a[15]),
+                           "r"(a[16]), "r"(a[17]), "r"(a[18]), "r"(a[19]), "r"(a[20]), "r"(a[21]), "r"(a[22]), "r"(a[23]),
+                           "r"(a[24]), "r"(a[25]), "r"(a[26]), "r"(a[27]), "r"(a[28]), "r"(a[29]), "r"(a[30]), "r"(a[31]) : "memory");
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&s_ready[wg][slot])) : "memory");
         }
-    }
-    const int my_iters = it;                                     // chunks this warpgroup issued (may be 0)
-    __syncthreads();                                             // s_sumx / s_sumxp visible; all MMAs issued
-
-    // ---- epilogue: warpgroup 0 adds the four accumulators of its rows in a fixed order
-    float v[kNB];
-#pragma unroll
-    for (int b = 0; b < kNB; ++b) v[b] = 0.f;
-    if (wg == 0) {
-        for (int w = 0; w < kWarpgroups; ++w) {
-            const int iters_w = (n_chunks > w) ? (n_chunks - w + kWarpgroups - 1) / kWarpgroups : 0;
-            if (iters_w == 0) continue;                          // that accumulator was never written
-            ok &= mbar_wait(smem_u32(&s_done[w]), 0);
+        if (wg == 0) {
+            // ---- epilogue: the accumulator of this thread's row
+            ok &= mbar_wait(smem_u32(&s_done), 0);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             uint32_t d[kNB];
-            const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + kAccCol + w * kNB;
+            const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + kAccCol;
             asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
                          : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
                            "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
                          : "r"(addr) : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int64_t row = row0 + row_l;
 #pragma unroll
-            for (int b = 0; b < kNB; ++b) v[b] += __uint_as_float(d[b]);
-        }
-        const int64_t row = row0 + row_l;
-#pragma unroll
-        for (int b = 0; b < kNB; ++b) {
-            if (b >= P.B) continue;
-            float val = v[b] - 128.0f * s_sumxp[b];
-            if (P.ovf_row_ptr && row < P.N) {                    // extra-precision columns: their field is one higher
-                const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
-                const int32_t pe = P.ovf_row_ptr[row + 1];
-                float ev = 0.f;
-                for (int32_t p = P.ovf_row_ptr[row] + split; p < pe; p += n_split) ev += __bfloat162float(xr[P.ovf_col[p]]);
-                val += ev;
-            }
-            if (n_split == 1) {
-                if (row < P.N) P.y[(int64_t)b * P.ldy + row] = a_pre * (val * (float)(1 << sh) - z_pre * s_sumx[b]);
-            } else {
-                s_part[row_l][b] = val;
+            for (int b = 0; b < kNB; ++b) {
+                if (b >= P.B) continue;
+                float val = __uint_as_float(d[b]) - 128.0f * s_sumxp[b];
+                if (P.ovf_row_ptr && row < P.N) {                // extra-precision columns: their field is one higher
+                    const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
+                    const int32_t pe = P.ovf_row_ptr[row + 1];
+                    float ev = 0.f;
+                    for (int32_t p = P.ovf_row_ptr[row] + split; p < pe; p += n_split) ev += __bfloat162float(xr[P.ovf_col[p]]);
+                    val += ev;
+                }
+                if (n_split == 1) {
+                    if (row < P.N) P.y[(int64_t)b * P.ldy + row] = a_pre * (val * (float)(1 << sh) - z_pre * s_sumx[b]);
+                } else {
+                    s_part[row_l][b] = val;
+                }
             }
         }
+        if (!ok) s_timeout = 1;
+    } else if (warp < kUnpackWarps + kStageWarps) {
+        // ================= stage warps: the only readers of x; everything after this point depends on the predecessor
+        if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+        const int st_tid = tid - 32 * kUnpackWarps;              // 0..127
+        const int bcol = st_tid & (kNB - 1);
+        const int64_t k_base = slice_off * 8 / R;
+        const bool wide = P.step_bytes == 512;
+        float sx = 0.f, sxp = 0.f;
+        if (wide || bcol < 8) {
+            for (int st = st_tid >> 4; st < n_steps; st += (32 * kStageWarps) / kNB) {
+                const int64_t k = k_base + (int64_t)st * kKPerStep;
+                uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
+                if (bcol < P.B && k < P.K) stage_step<R>(P.x + (int64_t)bcol * P.ldx + k, h0, h1, sx, sxp);
+                unsigned char* base = xs + (size_t)st * P.step_bytes + (wide ? (bcol >> 3) * 128 : 0) + (bcol & 7) * 16;
+                *reinterpret_cast<uint4*>(base) = h0;
+                *reinterpret_cast<uint4*>(base + (wide ? 256 : 128)) = h1;
+            }
+        }
+        sx += __shfl_xor_sync(0xffffffffu, sx, 16);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 16);
+        const int sw = warp - kUnpackWarps;
+        if (lane < kNB) { s_red[0][sw][lane] = sx; s_red[1][sw][lane] = sxp; }
+        asm volatile("bar.sync 1, 128;" ::: "memory");           // the four stage warps
+        if (st_tid < kNB) {
+            float a = 0.f, b = 0.f;
+            for (int w = 0; w < kStageWarps; ++w) { a += s_red[0][w][st_tid]; b += s_red[1][w][st_tid]; }
+            s_sumx[st_tid] = a;
+            s_sumxp[st_tid] = b;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // x' was written with ordinary stores, the MMA reads it
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&s_xready)) : "memory");
+    } else if (lane == 0) {
+        // ================= control lane: weight copies now, all MMAs later (in slot order)
+        for (int b = 0; b < n_boxes; ++b) {
+            const uint32_t bar = smem_u32(&s_wbar[b]);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBoxBytes) : "memory");
+            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                         ::"r"(smem_u32(wt + (size_t)b * kBoxBytes)), "l"(&tm_w), "r"((int)(slice_off + b * 128)), "r"((int)row0), "r"(bar) : "memory");
+        }
+        bool ok = mbar_wait(smem_u32(&s_xready), 0);
+        const uint32_t lbo = P.step_bytes == 512 ? 256u : 128u, sbo = P.step_bytes == 512 ? 128u : 0u;
+        for (int s = 0; s < n_slots && ok; ++s) {
+            const int wg = s & 1, it = s >> 1, slot = it % kSlots;
+            ok &= mbar_wait(smem_u32(&s_ready[wg][slot]), (uint32_t)(it / kSlots) & 1u);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = tmem + kSlotCol + (wg * kSlots + slot) * kSlotCols;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint64_t bd = b_desc(smem_u32(xs + (size_t)(4 * s + i) * P.step_bytes), lbo, sbo);
+                const uint32_t accumulate = (s > 0 || i > 0) ? 1u : 0u;
+                asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p; }"
+                             ::"r"(tmem + kAccCol), "r"(a_addr + i * 8), "l"(bd), "r"(kIdesc), "r"(accumulate) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_free[wg][slot])) : "memory");
+        }
+        // arrives when every MMA above has retired (also after a give-up, so the epilogue never waits in vain)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_done)) : "memory");
+        if (!ok) s_timeout = 1;
     }
-    (void)my_iters;
-    if (!ok && lane == 0) report(P.dev_status, MATQ_ERR_TIMEOUT);
 
     // ---- K slices: sum across the cluster in rank order
     if (n_split > 1) {
@@ -369,51 +366,85 @@ gemv_tcgen05(const Params P) {
         cluster.sync();                                          // peers may still be reading this CTA's tile
     }
 
-    // ---- release tensor memory (all tcgen05 traffic of this CTA has been waited for above)
+    // ---- release tensor memory (every tcgen05 operation of this CTA has been waited for above)
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (tid == 0 && s_timeout) report(P.dev_status, MATQ_ERR_TIMEOUT);
     if (warp == 0)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
-// Host side.  Returns MATQ_ERR_SHAPE when the call does not fit this kernel (the caller then uses another path).
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Returns MATQ_ERR_SHAPE when the call does not fit this kernel (the caller then uses another path).
 template <int R>
 inline int launch(const uint8_t* packed, int64_t N, int64_t K, const float* alpha, const float* zero,
                   const int32_t* ovf_row_ptr, const uint16_t* ovf_col, const void* x, int B, int64_t ldx,
                   float* y, int64_t ldy, int32_t* dev_status, bool pdl, cudaStream_t s) {
-    constexpr int kSlotBytes = 16 * 2 / Fmt<R>::kStepsPerChunk;
+    constexpr int kSlotBytes = 16 * 4 / Fmt<R>::kStepsPerChunk;
     Params P;
-    P.packed = packed; P.alpha = alpha; P.zero = zero; P.ovf_row_ptr = ovf_row_ptr; P.ovf_col = ovf_col;
+    P.alpha = alpha; P.zero = zero; P.ovf_row_ptr = ovf_row_ptr; P.ovf_col = ovf_col;
     P.x = static_cast<const __nv_bfloat16*>(x); P.y = y; P.dev_status = dev_status;
     P.N = N; P.K = K; P.ldx = ldx; P.ldy = ldy;
     P.row_bytes = K * R / 8;
     P.B = B;
+    P.step_bytes = B <= 8 ? 256 : 512;
     P.pdl = pdl ? 1 : 0;
+    if (P.row_bytes % 16 != 0 || P.row_bytes >= (1ll << 31) || N >= (1ll << 31)) return MATQ_ERR_SHAPE;
     const int64_t row_blocks = (N + kRows - 1) / kRows;
     const int sms = sm_count();
-    // shared memory per byte of row slice: 128 tile bytes + x' (512 bytes per step = per kSlotBytes / 2 row bytes)
     auto smem_for = [&](int64_t sb) {
-        return (size_t)kRows * (size_t)(((sb + 127) / 128) * 128 + 16) + (size_t)(sb / kSlotBytes) * 2 * kStepBytes;
+        const int64_t boxes = (sb + 127) / 128, slots = (sb + kSlotBytes - 1) / kSlotBytes;
+        return (size_t)(boxes * kBoxBytes + slots * 4 * P.step_bytes + 1024);
     };
-    int n_split = (int)((sms + row_blocks - 1) / row_blocks);     // about one CTA per SM
+    // slices of whole 128-byte boxes; about one CTA per SM, at most 8 slices (portable cluster), at most kMaxBoxes boxes
+    const int64_t total_boxes = (P.row_bytes + 127) / 128;
+    int n_split = (int)((sms + row_blocks - 1) / row_blocks);
     if (n_split < 1) n_split = 1;
     if (n_split > 8) n_split = 8;
+    if (n_split > total_boxes) n_split = (int)total_boxes;
     int64_t sb = 0;
     for (;; ++n_split) {
-        if (n_split > 8) return MATQ_ERR_SHAPE;
-        sb = ((P.row_bytes + n_split - 1) / n_split + 15) / 16 * 16;
-        if (smem_for(sb) <= 200 * 1024) break;
+        if (n_split > 8 || n_split > total_boxes) return MATQ_ERR_SHAPE;
+        sb = ((total_boxes + n_split - 1) / n_split) * 128;
+        if (sb / 128 <= kMaxBoxes && smem_for(sb) <= 200 * 1024) break;
     }
     n_split = (int)((P.row_bytes + sb - 1) / sb);
     P.slice_bytes = (int)sb;
-    P.tile_stride = (int)(((sb + 127) / 128) * 128 + 16);          // 16 mod 128: conflict-free 16-byte reads down a column of rows
+    CUtensorMap tm;
+    {
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return MATQ_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)P.row_bytes, (cuuint64_t)N};
+        const cuuint64_t strides[1] = {(cuuint64_t)P.row_bytes};
+        const cuuint32_t box[2] = {128, (cuuint32_t)kRows};
+        const cuuint32_t estr[2] = {1, 1};
+        if (fn(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(packed), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return MATQ_ERR_SHAPE;
+    }
     // At least 80 KB per CTA keeps residency at two CTAs per SM, which is what the 512 TMEM columns allow
     // (2 x 256): tcgen05.alloc then never has to wait for another CTA.
     const size_t smem = smem_for(sb) < 80 * 1024 ? 80 * 1024 : smem_for(sb);
     auto kern = gemv_tcgen05<R>;
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return MATQ_ERR_CUDA;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)row_blocks, (unsigned)n_split, 1);
     cfg.blockDim = dim3(kThreads);
@@ -433,7 +464,7 @@ inline int launch(const uint8_t* packed, int64_t N, int64_t K, const float* alph
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    if (cudaLaunchKernelEx(&cfg, kern, P) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
+    if (cudaLaunchKernelEx(&cfg, kern, tm, P) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
     return MATQ_OK;
 }
 

@@ -8,7 +8,9 @@
 //
 // The arithmetic of Eq. 1 is pinned to IEEE binary32 with one correctly
 // rounded operation per step (__fdiv_rn / __fadd_rn / __fsub_rn are never
-// contracted into FMAs), so the codes are reproducible bit for bit.
+// contracted into FMAs), so the codes are reproducible bit for bit.  The
+// register-resident kernel reaches the same bits through a cheaper sequence
+// with a proven guard band and falls back to the pinned sequence inside it.
 #include "common.cuh"
 
 namespace matq {
@@ -77,6 +79,49 @@ __device__ __forceinline__ uint32_t codes_from_words(uint32_t w0, uint32_t w1, f
     return c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
 }
 
+// ---- the same codes without the special-function pipe ---------------------------------------------------------
+// Per element the pinned arithmetic needs a division, a floor and a float->int conversion, all of which issue on
+// the quarter-rate special-function pipe and bound the kernel.  The fast path below produces the SAME codes:
+//   t1 = w * ra refined by one Newton step (ra = correctly rounded 1/alpha, once per row) is within one ulp of
+//        the correctly rounded quotient t;
+//   u1 = t1 + z is then within err = 2^-23 (2 |t| + |z|) of the pinned u;
+//   r  = u1 rounded to the nearest integer with the 1.5 * 2^23 trick (no conversion instruction).
+// Rounding half up and rounding to nearest agree unless u sits on a tie, and u and u1 round alike unless u1 is within
+// err of a tie.  So whenever |u1 - r| < 1/2 - delta (delta = 4 err, a per-row constant) r IS the pinned result;
+// otherwise (about one element in a thousand) the element is recomputed with the pinned sequence.
+struct RowFast {
+    float a, z, ra, tie_guard;   // tie_guard = 1/2 - delta; <= 0 sends every element down the pinned path
+};
+
+__device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx) {
+    RowFast f{a, z, 0.f, -1.f};
+    const float big = fmaxf(fabsf(mn), fabsf(mx));
+    if (a > 1e-30f && a < 1e30f && fabsf(z) < 1048576.0f && big < 1e30f) {
+        f.ra = __frcp_rn(a);
+        const float tmax = big * f.ra * 1.0001f;
+        const float delta = (2.0f * tmax + fabsf(z) + 1.0f) * 4.76837158e-7f;      // 4 * 2^-23 * (2 |t| + |z| + 1)
+        if (tmax + fabsf(z) < 2097152.0f) f.tie_guard = 0.5f - delta;              // |u| < 2^21: the rounding trick is exact
+    }
+    return f;
+}
+
+__device__ __forceinline__ uint32_t code_fast(float w, const RowFast& f) {
+    const float t0 = __fmul_rn(w, f.ra);
+    const float e = __fmaf_rn(-t0, f.a, w);
+    const float t1 = __fmaf_rn(e, f.ra, t0);
+    const float u1 = __fadd_rn(t1, f.z);
+    const float m = __fadd_rn(u1, 12582912.0f);                 // 1.5 * 2^23: the sum is u1 rounded to an integer
+    float r = __fsub_rn(m, 12582912.0f);
+    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) r = code_from_weight(w, f.a, f.z);   // near a tie (or NaN): pinned path
+    r = fminf(fmaxf(r, 0.0f), 255.0f);
+    return __float_as_uint(__fadd_rn(r, 12582912.0f)) & 0xffu;
+}
+
+__device__ __forceinline__ uint32_t codes_from_words_fast(uint32_t w0, uint32_t w1, const RowFast& f) {
+    return code_fast(__uint_as_float(w0 << 16), f) | (code_fast(__uint_as_float(w0 & 0xffff0000u), f) << 8) |
+           (code_fast(__uint_as_float(w1 << 16), f) << 16) | (code_fast(__uint_as_float(w1 & 0xffff0000u), f) << 24);
+}
+
 // Fast path: K % 16 == 0, rows 16-byte aligned.  Dynamic shared memory: K * 2 bytes.
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
@@ -117,6 +162,82 @@ quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
             }
         }
         __syncthreads();                           // row_s is reused by the next row
+    }
+}
+
+// Register-resident path (K <= 20480, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
+// (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
+// folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
+template <int NV>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw, int wpr,
+                  uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
+                  int32_t* dev_status) {
+    __shared__ float s_mn[kQuantThreads / 32], s_mx[kQuantThreads / 32];
+    __shared__ int s_bad[kQuantThreads / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rows_per_cta = (kQuantThreads / 32) / wpr;
+    const int team = warp / wpr, team_tid = (warp % wpr) * 32 + lane, team_threads = 32 * wpr;
+    const int nvec = K >> 3;
+    for (int64_t n_base = (int64_t)blockIdx.x * rows_per_cta; n_base < N; n_base += (int64_t)gridDim.x * rows_per_cta) {
+        const int64_t n = n_base + team;
+        const bool live = n < N;
+        uint4 v[NV];
+        float mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);
+        int bad = 0;
+        if (live) {
+            const uint4* src = reinterpret_cast<const uint4*>(W + n * ldw);
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                const int i = team_tid + j * team_threads;
+                if (i < nvec) v[j] = ld_stream_u4(src + i);
+            }
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                const int i = team_tid + j * team_threads;
+                if (i < nvec) {
+                    fold_word(v[j].x, mn, mx, bad);
+                    fold_word(v[j].y, mn, mx, bad);
+                    fold_word(v[j].z, mn, mx, bad);
+                    fold_word(v[j].w, mn, mx, bad);
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            bad |= __shfl_xor_sync(0xffffffffu, bad, o);
+        }
+        if (wpr > 1) {                                    // uniform over the CTA
+            __syncthreads();                              // the previous round's readers are done
+            if (lane == 0) { s_mn[warp] = mn; s_mx[warp] = mx; s_bad[warp] = bad; }
+            __syncthreads();
+            for (int w = 0; w < wpr; ++w) {
+                mn = fminf(mn, s_mn[team * wpr + w]);
+                mx = fmaxf(mx, s_mx[team * wpr + w]);
+                bad |= s_bad[team * wpr + w];
+            }
+        }
+        if (!live) continue;
+        RowRange rr{mn, mx, bad};
+        float a, z;
+        scale_zero(rr, a, z);
+        if (team_tid == 0) {
+            if (bad) report(dev_status, MATQ_ERR_NONFINITE);
+            alpha[n] = a;
+            zero[n] = z;
+        }
+        if (q) {
+            uint2* dst = reinterpret_cast<uint2*>(q + n * (int64_t)K);
+            const RowFast f = row_fast(a, z, mn, mx);
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                const int i = team_tid + j * team_threads;
+                if (i < nvec)
+                    dst[i] = make_uint2(codes_from_words_fast(v[j].x, v[j].y, f), codes_from_words_fast(v[j].z, v[j].w, f));
+            }
+        }
     }
 }
 
@@ -161,10 +282,28 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int sms = sm_count();
+    const uint16_t* Wb = static_cast<const uint16_t*>(W);
+    const bool reg = aligned16(W) && (K % 8 == 0) && (ldw % 8 == 0) && K <= 20480 &&
+                     (q == nullptr || (reinterpret_cast<uintptr_t>(q) & 7u) == 0);
     const bool fast = aligned16(W) && (K % 16 == 0) && (ldw % 8 == 0) && K <= 65536 &&
                       (q == nullptr || aligned16(q));
-    const int sms = sm_count();
-    if (fast) {
+    if (reg) {
+        const int nvec = (int)(K / 8);
+        int wpr = 1;
+        while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 10) wpr *= 2;
+        const int nv = (nvec + 32 * wpr - 1) / (32 * wpr);
+        const int rows_per_cta = 8 / wpr;
+        int64_t grid = (N + rows_per_cta - 1) / rows_per_cta;
+        if (grid > (int64_t)sms * 16) grid = (int64_t)sms * 16;
+#define MATQ_QUANT_REG(NV) quantize_rows_reg<NV><<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status)
+        if (nv <= 2) MATQ_QUANT_REG(2);
+        else if (nv <= 4) MATQ_QUANT_REG(4);
+        else if (nv <= 6) MATQ_QUANT_REG(6);
+        else if (nv <= 8) MATQ_QUANT_REG(8);
+        else MATQ_QUANT_REG(10);
+#undef MATQ_QUANT_REG
+    } else if (fast) {
         const size_t smem = (size_t)K * 2;
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(quantize_rows_vec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -172,12 +311,10 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
         int per_sm = (int)((200u * 1024u) / (smem + 1024));
         per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
         const int64_t grid = N < (int64_t)sms * per_sm ? N : (int64_t)sms * per_sm;
-        quantize_rows_vec<<<(unsigned)grid, kQuantThreads, smem, s>>>(
-            static_cast<const uint16_t*>(W), N, (int)K, ldw, q, alpha, zero, dev_status);
+        quantize_rows_vec<<<(unsigned)grid, kQuantThreads, smem, s>>>(Wb, N, (int)K, ldw, q, alpha, zero, dev_status);
     } else {
         const int64_t grid = N < (int64_t)sms * 8 ? N : (int64_t)sms * 8;
-        quantize_rows_generic<<<(unsigned)grid, kQuantThreads, 0, s>>>(
-            static_cast<const uint16_t*>(W), N, K, ldw, q, alpha, zero, dev_status);
+        quantize_rows_generic<<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, K, ldw, q, alpha, zero, dev_status);
     }
     return launch_status();
 }

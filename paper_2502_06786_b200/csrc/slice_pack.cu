@@ -103,6 +103,10 @@ slice_pack_generic(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, i
 }
 
 // row_ptr[n+1] holds row n's count on entry; on exit row_ptr is the exclusive scan.
+// One CTA: every thread scans kScanItems consecutive rows in registers, the 1024 thread totals are scanned once
+// through shared memory, and a running carry links passes of 1024 * kScanItems rows.
+constexpr int kScanItems = 16;
+
 __global__ void __launch_bounds__(1024)
 ovf_scan(int32_t* __restrict__ row_ptr, int64_t N, int64_t capacity, int64_t* __restrict__ total_out,
          int32_t* dev_status) {
@@ -111,9 +115,16 @@ ovf_scan(int32_t* __restrict__ row_ptr, int64_t N, int64_t capacity, int64_t* __
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) { carry_s = 0; row_ptr[0] = 0; }
     __syncthreads();
-    for (int64_t base = 0; base < N; base += 1024) {
-        const int64_t n = base + threadIdx.x;
-        int64_t v = (n < N) ? row_ptr[n + 1] : 0;
+    for (int64_t base = 0; base < N; base += 1024 * kScanItems) {
+        const int64_t n0 = base + (int64_t)threadIdx.x * kScanItems;
+        int32_t c[kScanItems];
+        int64_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i) {
+            c[i] = (n0 + i < N) ? row_ptr[n0 + i + 1] : 0;
+            mine += c[i];
+        }
+        int64_t v = mine;                                   // inclusive scan of the thread totals
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int64_t t = __shfl_up_sync(0xffffffffu, v, o);
@@ -131,11 +142,14 @@ ovf_scan(int32_t* __restrict__ row_ptr, int64_t N, int64_t capacity, int64_t* __
             warp_sum[lane] = w;
         }
         __syncthreads();
-        const int64_t carry = carry_s;
-        const int64_t incl = carry + v + (warp ? warp_sum[warp - 1] : 0);
-        if (n < N) row_ptr[n + 1] = (int32_t)(incl > 0x7fffffff ? 0x7fffffff : incl);
+        int64_t run = carry_s + (v - mine) + (warp ? warp_sum[warp - 1] : 0);   // sum of everything before row n0
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i) {
+            run += c[i];
+            if (n0 + i < N) row_ptr[n0 + i + 1] = (int32_t)(run > 0x7fffffff ? 0x7fffffff : run);
+        }
         __syncthreads();
-        if (threadIdx.x == 1023) carry_s = incl;
+        if (threadIdx.x == 1023) carry_s = run;
         __syncthreads();
     }
     if (threadIdx.x == 0) {

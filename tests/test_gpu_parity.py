@@ -58,6 +58,26 @@ def test_quantize_special_rows_and_strided_input():
     assert q3 is None and np.array_equal(host(a3), a_ref) and np.array_equal(host(z3), z_ref)
 
 
+def test_quantize_bit_exact_over_many_scales_and_offsets():
+    # Rows with very different ranges and offsets: zero-centred, same-sign (z far outside [0, 255], up to the point where
+    # the kernel must leave its fast path), tiny and huge scales, and many exact ties (weights on a coarse grid).
+    rng = np.random.default_rng(123)
+    N, K = 4096, 512
+    base = synth.bf16_bits_to_f32(synth.normal_bf16((N, K), 1.0, 314)).astype(np.float64)
+    scale = 10.0 ** rng.uniform(-6, 4, size=(N, 1))
+    offset = np.where(rng.random((N, 1)) < 0.5, 0.0, 10.0 ** rng.uniform(-2, 7, size=(N, 1))) * scale
+    Wf = base * scale + offset
+    Wf[::7] = np.round(base[::7] * 8) / 8                 # coarse grid: u lands on exact halves often
+    Wf[::11] = np.round(base[::11] * 2) * 0.5 + 1000.0
+    W = synth.f32_to_bf16_bits(Wf.astype(np.float32))
+    st, q_ref, a_ref, z_ref = ref.quantize(W)
+    assert st == ref.OK
+    q, a, z = mq.quantize(bf16_dev(W))
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert np.array_equal(host(q), q_ref)
+    assert np.abs(z_ref).max() > 2 ** 21                   # some rows did take the pinned path
+
+
 def test_quantize_reports_nonfinite_without_trapping():
     Wf = synth.bf16_bits_to_f32(synth.normal_bf16((4, 128), 0.02, 9)).copy()
     Wf[2, 77] = np.inf
