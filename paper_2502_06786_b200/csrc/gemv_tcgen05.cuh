@@ -20,13 +20,14 @@
 // in the epilogue with the separately accumulated sum.
 //
 // Warp roles (13 warps):
-//   warps 0-7   two "unpack" warpgroups.  Each owns three TMEM slots of 32 columns (4 instructions' worth of A) and
+//   warps 0-7   two "unpack" warpgroups.  Each owns two TMEM slots of 32 columns (4 instructions' worth of A) and
 //               fills them round-robin from the shared-memory weight tile; an mbarrier per slot says "ready", the
 //               tcgen05.commit of the instructions that read a slot says "free".  They start as soon as the weights
 //               land, i.e. BEFORE the kernel's predecessor in the stream has finished.
 //   warps 8-11  wait for the predecessor (programmatic dependent launch), stage x' and the two sums, signal "x ready".
 //   warp 12     one lane issues the TMA copies of the weight tile (before the dependency wait) and later all MMAs,
-//               always in slot order, so the single accumulator is summed in a fixed order (deterministic results).
+//               always in slot order and round-robin over eight accumulators (a fixed assignment, so results are
+//               reproducible); one accumulator alone would serialise the tiny N = 16 instructions on their latency.
 //
 // Data movement.  The CTA's slice of the packed plane is fetched as 128-byte x 128-row boxes of a 2-D tensor map over
 // the plane (uint8, 128-byte swizzle so that 32 rows can be read 16 bytes at a time without bank conflicts; rows and
@@ -48,9 +49,11 @@ constexpr int kThreads = 32 * (kUnpackWarps + kStageWarps + 1);
 constexpr int kRows = 128;                   // M of the MMA = TMEM lanes
 constexpr int kNB = 16;                      // N of the MMA = batch columns (padded)
 constexpr int kSlotCols = 32;                // TMEM columns of one A slot = four K = 16 instructions
-constexpr int kSlots = 3;                    // slots per unpack warpgroup
-constexpr int kTmemCols = 256;               // accumulator 16 + 2 warpgroups x 3 slots x 32 = 208 -> 256
-constexpr int kAccCol = 0, kSlotCol = 32;
+constexpr int kSlots = 2;                    // slots per unpack warpgroup
+constexpr int kAccs = 8;                     // independent accumulators: consecutive MMAs into ONE accumulator would
+                                             // each wait out the previous one's full latency (N = 16 is a tiny instruction)
+constexpr int kTmemCols = 256;               // 8 accumulators x 16 + 2 warpgroups x 2 slots x 32 = 256
+constexpr int kAccCol = 0, kSlotCol = kAccs * kNB;
 constexpr int kBoxBytes = 128 * kRows;       // one TMA box: 128 bytes of 128 rows
 constexpr int kMaxBoxes = 8;
 constexpr uint32_t kSpinLimit = 1u << 22;    // mbarrier polls before a wait gives up
@@ -259,18 +262,26 @@ gemv_tcgen05(const __grid_constant__ CUtensorMap tm_w, const Params P) {
             // ---- epilogue: the accumulator of this thread's row
             ok &= mbar_wait(smem_u32(&s_done), 0);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            uint32_t d[kNB];
-            const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + kAccCol;
-            asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
-                           "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
-                         : "r"(addr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            float acc[kNB];
+#pragma unroll
+            for (int b = 0; b < kNB; ++b) acc[b] = 0.f;
+            const int used = n_steps < kAccs ? n_steps : kAccs;  // accumulators that were written at all
+            for (int a = 0; a < used; ++a) {                     // fixed order: results are reproducible
+                uint32_t d[kNB];
+                const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + kAccCol + a * kNB;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                             : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
+                               "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
+                             : "r"(addr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int b = 0; b < kNB; ++b) acc[b] += __uint_as_float(d[b]);
+            }
             const int64_t row = row0 + row_l;
 #pragma unroll
             for (int b = 0; b < kNB; ++b) {
                 if (b >= P.B) continue;
-                float val = __uint_as_float(d[b]) - 128.0f * s_sumxp[b];
+                float val = acc[b] - 128.0f * s_sumxp[b];
                 if (P.ovf_row_ptr && row < P.N) {                // extra-precision columns: their field is one higher
                     const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
                     const int32_t pe = P.ovf_row_ptr[row + 1];
@@ -326,6 +337,10 @@ gemv_tcgen05(const __grid_constant__ CUtensorMap tm_w, const Params P) {
         }
         bool ok = mbar_wait(smem_u32(&s_xready), 0);
         const uint32_t lbo = P.step_bytes == 512 ? 256u : 128u, sbo = P.step_bytes == 512 ? 128u : 0u;
+        // descriptor of step 0; later steps only move the start address (14-bit field in units of 16 bytes)
+        uint64_t bd = b_desc(smem_u32(xs), lbo, sbo);
+        const uint64_t bd_step = (uint64_t)(P.step_bytes >> 4);
+        int n_mma = 0;                                            // MMA number n accumulates into accumulator n % kAccs
         for (int s = 0; s < n_slots && ok; ++s) {
             const int wg = s & 1, it = s >> 1, slot = it % kSlots;
             ok &= mbar_wait(smem_u32(&s_ready[wg][slot]), (uint32_t)(it / kSlots) & 1u);
@@ -334,10 +349,11 @@ gemv_tcgen05(const __grid_constant__ CUtensorMap tm_w, const Params P) {
             const uint32_t a_addr = tmem + kSlotCol + (wg * kSlots + slot) * kSlotCols;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint64_t bd = b_desc(smem_u32(xs + (size_t)(4 * s + i) * P.step_bytes), lbo, sbo);
-                const uint32_t accumulate = (s > 0 || i > 0) ? 1u : 0u;
                 asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p; }"
-                             ::"r"(tmem + kAccCol), "r"(a_addr + i * 8), "l"(bd), "r"(kIdesc), "r"(accumulate) : "memory");
+                             ::"r"(tmem + kAccCol + (n_mma % kAccs) * kNB), "r"(a_addr + i * 8), "l"(bd), "r"(kIdesc),
+                               "r"(n_mma >= kAccs ? 1u : 0u) : "memory");
+                ++n_mma;
+                bd += bd_step;
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_free[wg][slot])) : "memory");
         }
