@@ -105,6 +105,10 @@ __device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx
     return f;
 }
 
+// Out of line on purpose: inlined, the compiler predicates the whole pinned sequence into the fast path and every
+// element pays for it; as a call it costs nothing unless a lane really is near a tie.
+__device__ __noinline__ float code_pinned(float w, float a, float z) { return code_from_weight(w, a, z); }
+
 __device__ __forceinline__ uint32_t code_fast(float w, const RowFast& f) {
     const float t0 = __fmul_rn(w, f.ra);
     const float e = __fmaf_rn(-t0, f.a, w);
@@ -112,7 +116,7 @@ __device__ __forceinline__ uint32_t code_fast(float w, const RowFast& f) {
     const float u1 = __fadd_rn(t1, f.z);
     const float m = __fadd_rn(u1, 12582912.0f);                 // 1.5 * 2^23: the sum is u1 rounded to an integer
     float r = __fsub_rn(m, 12582912.0f);
-    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) r = code_from_weight(w, f.a, f.z);   // near a tie (or NaN): pinned path
+    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) r = code_pinned(w, f.a, f.z);        // near a tie (or NaN): pinned path
     r = fminf(fmaxf(r, 0.0f), 255.0f);
     return __float_as_uint(__fadd_rn(r, 12582912.0f)) & 0xffu;
 }
@@ -165,7 +169,15 @@ quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
     }
 }
 
-// Register-resident path (K <= 20480, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
+// Range of two bf16 values at a time: packed min / max (NaN operands are ignored, as fminf / fmaxf do) and a packed
+// "exponent all ones" detector: |v| + 0x0080 carries into bit 15 exactly when |v| >= 0x7f80 (Inf or NaN).
+__device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& mx2, uint32_t& bad2) {
+    asm("min.bf16x2 %0, %0, %1;" : "+r"(mn2) : "r"(w));
+    asm("max.bf16x2 %0, %0, %1;" : "+r"(mx2) : "r"(w));
+    bad2 |= (w & 0x7fff7fffu) + 0x00800080u;
+}
+
+// Register-resident path (K <= 16384, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
 // (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
 // folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
 template <int NV>
@@ -183,8 +195,7 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
         const int64_t n = n_base + team;
         const bool live = n < N;
         uint4 v[NV];
-        float mn = __int_as_float(0x7f800000), mx = __int_as_float(0xff800000);
-        int bad = 0;
+        uint32_t mn2 = 0x7f807f80u, mx2 = 0xff80ff80u, bad2 = 0;      // +Inf / -Inf pairs
         if (live) {
             const uint4* src = reinterpret_cast<const uint4*>(W + n * ldw);
 #pragma unroll
@@ -196,13 +207,16 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
             for (int j = 0; j < NV; ++j) {
                 const int i = team_tid + j * team_threads;
                 if (i < nvec) {
-                    fold_word(v[j].x, mn, mx, bad);
-                    fold_word(v[j].y, mn, mx, bad);
-                    fold_word(v[j].z, mn, mx, bad);
-                    fold_word(v[j].w, mn, mx, bad);
+                    fold_word2(v[j].x, mn2, mx2, bad2);
+                    fold_word2(v[j].y, mn2, mx2, bad2);
+                    fold_word2(v[j].z, mn2, mx2, bad2);
+                    fold_word2(v[j].w, mn2, mx2, bad2);
                 }
             }
         }
+        float mn = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xffff0000u));
+        float mx = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xffff0000u));
+        int bad = (bad2 & 0x80008000u) != 0;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
@@ -284,24 +298,24 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int sms = sm_count();
     const uint16_t* Wb = static_cast<const uint16_t*>(W);
-    const bool reg = aligned16(W) && (K % 8 == 0) && (ldw % 8 == 0) && K <= 20480 &&
+    const bool reg = aligned16(W) && (K % 8 == 0) && (ldw % 8 == 0) && K <= 16384 &&
                      (q == nullptr || (reinterpret_cast<uintptr_t>(q) & 7u) == 0);
     const bool fast = aligned16(W) && (K % 16 == 0) && (ldw % 8 == 0) && K <= 65536 &&
                       (q == nullptr || aligned16(q));
     if (reg) {
         const int nvec = (int)(K / 8);
         int wpr = 1;
-        while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 10) wpr *= 2;
+        while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 5) wpr *= 2;
         const int nv = (nvec + 32 * wpr - 1) / (32 * wpr);
         const int rows_per_cta = 8 / wpr;
         int64_t grid = (N + rows_per_cta - 1) / rows_per_cta;
         if (grid > (int64_t)sms * 16) grid = (int64_t)sms * 16;
 #define MATQ_QUANT_REG(NV) quantize_rows_reg<NV><<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status)
         if (nv <= 2) MATQ_QUANT_REG(2);
+        else if (nv <= 3) MATQ_QUANT_REG(3);
         else if (nv <= 4) MATQ_QUANT_REG(4);
-        else if (nv <= 6) MATQ_QUANT_REG(6);
-        else if (nv <= 8) MATQ_QUANT_REG(8);
-        else MATQ_QUANT_REG(10);
+        else if (nv <= 5) MATQ_QUANT_REG(5);
+        else MATQ_QUANT_REG(8);
 #undef MATQ_QUANT_REG
     } else if (fast) {
         const size_t smem = (size_t)K * 2;
