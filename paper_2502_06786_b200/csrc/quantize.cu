@@ -82,9 +82,9 @@ __device__ __forceinline__ uint32_t codes_from_words(uint32_t w0, uint32_t w1, f
 // ---- the same codes without the special-function pipe ---------------------------------------------------------
 // Per element the pinned arithmetic needs a division, a floor and a float->int conversion, all of which issue on
 // the quarter-rate special-function pipe and bound the kernel.  The fast path below produces the SAME codes:
-//   t1 = w * ra refined by one Newton step (ra = correctly rounded 1/alpha, once per row) is within one ulp of
-//        the correctly rounded quotient t;
-//   u1 = t1 + z is then within err = 2^-23 (2 |t| + |z|) of the pinned u;
+//   u1 = fma(w, ra, z) with ra = correctly rounded 1/alpha (once per row): w * ra is within 2^-24 |t| of the exact
+//        quotient and the sum is rounded once, so u1 is within err = 2^-23 (2 |t| + |z|) of the pinned
+//        u = RN(RN(w / alpha) + z);
 //   r  = u1 rounded to the nearest integer with the 1.5 * 2^23 trick (no conversion instruction).
 // Rounding half up and rounding to nearest agree unless u sits on a tie, and u and u1 round alike unless u1 is within
 // err of a tie.  So whenever |u1 - r| < 1/2 - delta (delta = 4 err, a per-row constant) r IS the pinned result;
@@ -110,15 +110,12 @@ __device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx
 __device__ __noinline__ float code_pinned(float w, float a, float z) { return code_from_weight(w, a, z); }
 
 __device__ __forceinline__ uint32_t code_fast(float w, const RowFast& f) {
-    const float t0 = __fmul_rn(w, f.ra);
-    const float e = __fmaf_rn(-t0, f.a, w);
-    const float t1 = __fmaf_rn(e, f.ra, t0);
-    const float u1 = __fadd_rn(t1, f.z);
+    const float u1 = __fmaf_rn(w, f.ra, f.z);                   // within err of the pinned u (see above)
     const float m = __fadd_rn(u1, 12582912.0f);                 // 1.5 * 2^23: the sum is u1 rounded to an integer
-    float r = __fsub_rn(m, 12582912.0f);
-    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) r = code_pinned(w, f.a, f.z);        // near a tie (or NaN): pinned path
-    r = fminf(fmaxf(r, 0.0f), 255.0f);
-    return __float_as_uint(__fadd_rn(r, 12582912.0f)) & 0xffu;
+    const float r = __fsub_rn(m, 12582912.0f);
+    int code = __float_as_int(m) - 0x4b400000;                  // that integer, straight from the mantissa
+    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) code = (int)code_pinned(w, f.a, f.z);   // near a tie (or NaN): pinned path
+    return (uint32_t)min(max(code, 0), 255);
 }
 
 __device__ __forceinline__ uint32_t codes_from_words_fast(uint32_t w0, uint32_t w1, const RowFast& f) {
