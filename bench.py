@@ -346,11 +346,14 @@ def run_cuda(args, rank, world, local_rank):
     e2e = e2e_leg(st, plan, W_host, x_host, args, torch, world, dist if world > 1 else None)
 
     cfg4 = None
+    extras = {}
     if st.has_gemm and world == 1 and not args.no_cfg4:
         for t in (st.W, st.q, st.p4, st.p2):       # free the stack's large buffers first
             t.clear()
         torch.cuda.empty_cache()
         cfg4 = gemm_cfg4(mq, torch, peaks)
+        torch.cuda.empty_cache()
+        extras = {"gemv_cfg3": gemv_cfg3(mq, torch, peaks), "gemm_multi_cfg5_prefill": gemm_cfg5_prefill(mq, torch, peaks)}
 
     out = None
     if rank == 0:
@@ -370,6 +373,7 @@ def run_cuda(args, rank, world, local_rank):
         }
         if cfg4 is not None:
             out["gemm_multi_cfg4"] = cfg4
+        out.update(extras)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -402,6 +406,74 @@ def gemm_cfg4(mq, torch, peaks, reps=5):
             "roofline": {"kernel": "gemm_multi (quantize + expand + rowsum + tcgen05 GEMM)", "bound": "tensor", "achieved": round(tf, 1),
                          "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s", "frac": round(tf / peaks["bf16_tflops_sustained"], 4),
                          "traffic": None, "peak_source": peaks["source"] + " (sustained)"}}
+
+
+def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
+    """configs[2] shapes: Gemma-2-9B decoder layers (q, k, v, o, gate, up, down), B = 1, r = 4 and r = 2.  The planes are
+    random bytes (the kernels' speed does not depend on the field values); every matrix has its own buffers."""
+    shapes = [(n, k) for _ in range(layers) for (_, n, k) in synth.gemma2_9b_decoder_layer()]
+    out = {"workload": f"configs[2] Gemma-2-9B decoder layer shapes x {layers} layers, B = 1, one CUDA graph per precision, PDL"}
+    for r in (4, 2):
+        planes = [torch.randint(0, 256, (n, k * r // 8), dtype=torch.uint8, device="cuda") for n, k in shapes]
+        xs = [torch.randn(1, k, device="cuda").to(torch.bfloat16) for n, k in shapes]
+        ys = [torch.empty(1, n, device="cuda") for n, k in shapes]
+        al = [torch.ones(n, device="cuda") for n, k in shapes]
+
+        def run():
+            for i, (n, k) in enumerate(shapes):
+                mq.gemv(planes[i], k, r, al[i], al[i], xs[i], y=ys[i], flags=mq.GEMV_AUTO | mq.GEMV_PDL)
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            run()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                run()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            g.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        nbytes = sum(bytes_gemv(n, k, r, 1) for n, k in shapes)
+        out[f"r{r}_b1"] = {"ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
+                           "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4), "launches": len(shapes)}
+        del planes, xs, ys, al, g
+        torch.cuda.empty_cache()
+    return out
+
+
+def gemm_cfg5_prefill(mq, torch, peaks, reps=3):
+    """configs[4] prefill: extra-precision int2 plane (+ overflow lists, 5 % of the codes in the extra bucket) of a
+    Gemma-2-9B gate matrix (14336 x 3584), M = 2048 tokens, matq_gemm_multi(MATQ_SRC_PACKED)."""
+    N, K, M = 14336, 3584, 2048
+    q = torch.from_numpy(synth.skewed_codes((N, K), 0.05, 224, synth.seed_for(5, 0))).cuda()
+    sp = mq.slice_pack(q, 2, extra_precision=True, ovf_capacity=N * K // 8)
+    X = torch.from_numpy(synth.normal_bf16((M, K), 1.0, synth.seed_for(5, 500))).cuda().view(torch.bfloat16)
+    a = torch.full((N,), 1e-3, dtype=torch.float32, device="cuda"); z = torch.full((N,), 128.0, dtype=torch.float32, device="cuda")
+    Y = [torch.empty((M, N), dtype=torch.float32, device="cuda")]
+    ws = torch.empty(mq.gemm_multi_workspace_bytes(mq.SRC_PACKED, M, N, K, 1), dtype=torch.uint8, device="cuda")
+
+    def run():
+        mq.gemm_multi(mq.SRC_PACKED, sp["packed"], K, X, rs=(2,), alpha=a, zero=z, extra_precision=True,
+                      ovf_row_ptr=sp["ovf_row_ptr"], ovf_col=sp["ovf_col"], Ys=Y, workspace=ws)
+    run(); run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+    return {"workload": "configs[4] prefill: E.P. int2 plane + overflow lists, 14336x3584, M = 2048, one matq_gemm_multi(MATQ_SRC_PACKED) call",
+            "ms": round(ms, 3), "TFLOPs": round(tf, 1), "frac_tensor_sustained": round(tf / peaks["bf16_tflops_sustained"], 4),
+            "overflow_fraction": round(int(sp["ovf_count"].item()) / (N * K), 4)}
 
 
 def e2e_leg(st, plan, W_host, x_host, args, torch, world, dist):
