@@ -233,15 +233,31 @@ expand_codes(const uint4* __restrict__ q, int64_t nchunks, ExpandArgs A) {
     }
 }
 
-// packed r-bit plane -> bf16 plane of fields.  One thread = one 32-bit word of the plane.
+// packed r-bit plane -> bf16 plane of fields.  One thread = 16 bytes of the plane (128 / r fields), written as
+// 16-byte stores of eight bf16 each.
+template <int R>
 __global__ void __launch_bounds__(256)
-expand_packed(const uint32_t* __restrict__ packed, int64_t nwords, int r, __nv_bfloat16* __restrict__ plane) {
-    const int per = 32 / r;
-    const uint32_t mask = (1u << r) - 1u;
+expand_packed(const uint4* __restrict__ packed, int64_t nvec, __nv_bfloat16* __restrict__ plane) {
+    constexpr int kPerWord = 32 / R;
+    constexpr uint32_t kMask = (1u << R) - 1u;
     const int64_t stride = (int64_t)gridDim.x * 256;
-    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < nwords; i += stride) {
-        const uint32_t w = packed[i];
-        for (int f = 0; f < per; ++f) plane[i * per + f] = __float2bfloat16_rn((float)((w >> (f * r)) & mask));
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < nvec; i += stride) {
+        const uint4 v = ld_stream_u4(packed + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint4* dst = reinterpret_cast<uint4*>(plane + i * (4 * kPerWord));
+#pragma unroll
+        for (int t = 0; t < (4 * kPerWord) / 8; ++t) {         // eight fields per 16-byte store
+            uint32_t o[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const int e0 = 8 * t + 2 * h, e1 = e0 + 1;
+                const uint32_t lo = (w[e0 / kPerWord] >> ((e0 % kPerWord) * R)) & kMask;
+                const uint32_t hi = (w[e1 / kPerWord] >> ((e1 % kPerWord) * R)) & kMask;
+                o[h] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)lo)) |
+                       ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)hi)) << 16);
+            }
+            dst[t] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
     }
 }
 
@@ -396,10 +412,13 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
         if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
         expand_codes<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const uint4*>(codes), nchunks, EA);
     } else {
-        const int64_t nwords = N * K * rs[0] / 32;
-        int64_t blocks = (nwords + 255) / 256;
+        const int64_t nvec = N * K * rs[0] / 128;            // K % 64 == 0: rows are whole 16-byte pieces for r = 8, 4, 2
+        int64_t blocks = (nvec + 255) / 256;
         if (blocks > (int64_t)sms * 16) blocks = (int64_t)sms * 16;
-        expand_packed<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const uint32_t*>(Wsrc), nwords, rs[0], EA.plane[0]);
+        const uint4* pk = static_cast<const uint4*>(Wsrc);
+        if (rs[0] == 8) expand_packed<8><<<(unsigned)blocks, 256, 0, s>>>(pk, nvec, EA.plane[0]);
+        else if (rs[0] == 4) expand_packed<4><<<(unsigned)blocks, 256, 0, s>>>(pk, nvec, EA.plane[0]);
+        else expand_packed<2><<<(unsigned)blocks, 256, 0, s>>>(pk, nvec, EA.plane[0]);
         if (extra_precision && ovf_row_ptr) {
             int64_t b2 = (N + 7) / 8;
             if (b2 > (int64_t)sms * 16) b2 = (int64_t)sms * 16;
