@@ -68,7 +68,10 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t n0 = (int64_t)blockIdx.x * kBN, m0 = (int64_t)blockIdx.y * kBM;
+    // blockIdx.x walks the token tiles: CTAs that run together share one 128-channel slab of the planes (3 x 1 MB,
+    // read from HBM once) and differ in their X tiles, and all of X stays in the L2.  The other order re-streams the
+    // planes from HBM once per token tile.
+    const int64_t m0 = (int64_t)blockIdx.x * kBM, n0 = (int64_t)blockIdx.y * kBN;
     const int nkb = (int)(P.K / kBK);
     const int stage_bytes = (1 + P.n_r) * kTileBytes;
     const int tmem_cols = P.n_r == 1 ? 128 : (P.n_r == 2 ? 256 : 512);
@@ -452,7 +455,7 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     if (cudaFuncSetAttribute(gemm_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
-    const dim3 grid((unsigned)((N + kBN - 1) / kBN), (unsigned)((M + kBM - 1) / kBM), 1);
+    const dim3 grid((unsigned)((M + kBM - 1) / kBM), (unsigned)((N + kBN - 1) / kBN), 1);
     gemm_multi_kernel<<<grid, kThreads, smem, s>>>(tm_x, tm_b[0], tm_b[1], tm_b[2], P);
     return launch_status();
 }
