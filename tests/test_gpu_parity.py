@@ -116,7 +116,7 @@ def test_pack_bit_exact(r, N, K):
 
 @pytest.mark.parametrize("r", [4, 2])
 @pytest.mark.parametrize("N,K,p", [(64, 2304, 0.05), (1500, 512, 0.125), (9, 1000, 0.3), (40, 4096, 0.0), (33, 16384, 0.05),
-                                   (17, 9216, 0.5), (12, 32768, 0.02), (10, 16, 0.3)])
+                                   (17, 9216, 0.5), (12, 32768, 0.02), (10, 16, 0.3), (9216, 2304, 0.005), (4099, 256, 0.1)])
 def test_extra_precision_lists_bit_exact(r, N, K, p):
     q = synth.skewed_codes((N, K), p, 224, 400 + N) if p > 0 else synth.uniform_codes((N, K), 1) // 2
     if N > 8:
