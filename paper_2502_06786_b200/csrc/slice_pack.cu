@@ -263,26 +263,29 @@ ovf_fill_batched(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, con
 // Extra precision in ONE pass (K % 16 == 0, K <= 16384, N * K < 2^31): pack, count, scan and list in the same kernel,
 // so the codes are read from HBM once.
 //
-// A tile is eight consecutive rows, one warp per row.  The warp slices and packs its row, parks the 16-bit overflow
-// mask of every 16-code chunk in shared memory and counts the row's overflow elements.  Warp 0 then turns the eight
-// counts into the tile's place in the global list by a chained scan with look-back: the tile publishes its own total
-// ("partial") at once, sums the partials of the tiles before it until it meets one that already knows its inclusive
-// prefix, and finally replaces its own partial by its inclusive prefix.  With the place known every warp writes its
-// row's columns from the parked masks.
+// A tile is T = warps * rows_per_warp consecutive rows, sized on the host so that the matrix is about one tile per
+// SM.  Every warp slices and packs its rows, parks the 16-bit overflow mask of every 16-code chunk in shared memory
+// and counts each row's overflow elements.  Warp 0 scans the T counts and finds the tile's place in the global list
+// by a chained scan with look-back: the tile publishes its own total ("partial") at once, sums the partials of the
+// tiles before it until it meets one that already knows its inclusive prefix, and finally replaces its own partial
+// by its inclusive prefix.  With the place known every warp writes its rows' entries of ovf_row_ptr and their
+// columns from the parked masks.  Few, large tiles keep the look-back short (at most a few hundred flags, fetched
+// 128 at a time) while the other warps wait at a barrier without issuing anything.
 //
 // The scan state lives in ovf_row_ptr itself: the entry after a tile's last row is that tile's flag word,
 //   0xffffffff (the memset before the launch)  nothing yet
-//   0x80000000 | total of the tile             partial (a tile holds at most 8 * 16384 elements)
+//   0x80000000 | total of the tile             partial (a tile holds fewer than 2^30 elements)
 //   value < 2^31                               inclusive prefix = the final content of that entry
 //   0xc0000000                                 a wait gave up in this tile or before it
 // so value and state travel in one 32-bit word and no ordering between separate words is needed.  CTAs are
 // persistent and all resident (the grid is sized from the occupancy), tile t belongs to CTA t mod gridDim.x and only
 // ever waits for tiles below t, so every wait ends; each one is bounded all the same, and a wait that gives up
 // poisons the flags after it and reports MATQ_ERR_TIMEOUT instead of hanging.
-constexpr int kEpRows = 8;
 constexpr uint32_t kEpNothing = 0xffffffffu, kEpPartial = 0x80000000u, kEpPoison = 0xc0000000u;
 constexpr int kEpSpinLimit = 1 << 20;
 constexpr int kEpWindows = 4;              // look-back windows of 32 tiles fetched per round trip
+constexpr size_t kEpSmemLimit = 160 * 1024;
+constexpr int kEpBatch = 6;                // 16-byte loads a lane has in flight
 
 __device__ __forceinline__ uint32_t ld_flag(const uint32_t* p) {
     uint32_t v;
@@ -299,67 +302,77 @@ __device__ __forceinline__ uint32_t chunk_mask(const Sliced& s0, const Sliced& s
 }
 
 template <int PACK_R>
-__global__ void __launch_bounds__(kEpRows * 32)
-slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, uint8_t* __restrict__ packed,
-              uint8_t* __restrict__ sliced, uint32_t* __restrict__ row_ptr, uint16_t* __restrict__ ovf_col,
-              int64_t capacity, int64_t* __restrict__ total_out, int32_t* dev_status) {
-    extern __shared__ uint16_t ep_mask[];              // [kEpRows][K / 16]
-    __shared__ int row_cnt[kEpRows];
-    __shared__ uint32_t tile_base_s;
-    __shared__ int tile_bad_s;
+__global__ void __launch_bounds__(1024)
+slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, int rows_per_warp,
+              uint8_t* __restrict__ packed, uint8_t* __restrict__ sliced, uint32_t* __restrict__ row_ptr,
+              uint16_t* __restrict__ ovf_col, int64_t capacity, int64_t* __restrict__ total_out, int32_t* dev_status) {
+    extern __shared__ __align__(16) uint8_t ep_smem[];
+    __shared__ uint32_t base_s, total_s;
+    __shared__ int bad_s;
     const int r = PACK_R ? PACK_R : r_runtime;
     const int sh = kCodeBits - r;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int T = nwarps * rows_per_warp;              // rows per tile
     const int cpr = K / 16;                            // 16-code chunks per row
-    const int64_t ntiles = (N + kEpRows - 1) / kEpRows;
-    uint16_t* mrow = ep_mask + warp * cpr;
+    int* row_off = reinterpret_cast<int*>(ep_smem);    // [T] counts, then exclusive offsets within the tile
+    uint16_t* ep_mask = reinterpret_cast<uint16_t*>(row_off + T);   // [T][cpr]
+    const int64_t ntiles = (N + T - 1) / T;
     for (int64_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
-        const int64_t n = t * kEpRows + warp;
-        int cnt = 0;
-        if (n < N) {
-            const uint4* src = reinterpret_cast<const uint4*>(q + n * K);
-            const int64_t c_row = n * cpr;
-            for (int c0 = 0; c0 < cpr; c0 += 4 * 32) {
-                uint4 v[4];
+        const int64_t row0 = t * T;
+        for (int i = 0; i < rows_per_warp; ++i) {
+            const int lr = i * nwarps + warp;
+            const int64_t n = row0 + lr;
+            int cnt = 0;
+            if (n < N) {
+                const uint4* src = reinterpret_cast<const uint4*>(q + n * K);
+                const int64_t c_row = n * cpr;
+                uint16_t* mrow = ep_mask + (size_t)lr * cpr;
+                for (int c0 = 0; c0 < cpr; c0 += kEpBatch * 32) {
+                    uint4 v[kEpBatch];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + u * 32 + lane;
-                    v[u] = make_uint4(0, 0, 0, 0);
-                    if (c < cpr) v[u] = ld_stream_u4(src + c);
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + u * 32 + lane;
-                    if (c >= cpr) continue;
-                    const Sliced s0 = slice4(v[u].x, r), s1 = slice4(v[u].y, r), s2 = slice4(v[u].z, r), s3 = slice4(v[u].w, r);
-                    if (PACK_R == 4) {
-                        reinterpret_cast<uint2*>(packed)[c_row + c] =
-                            make_uint2(pack4<4>(s0.k) | (pack4<4>(s1.k) << 16), pack4<4>(s2.k) | (pack4<4>(s3.k) << 16));
-                    } else if (PACK_R == 2) {
-                        reinterpret_cast<uint32_t*>(packed)[c_row + c] =
-                            pack4<2>(s0.k) | (pack4<2>(s1.k) << 8) | (pack4<2>(s2.k) << 16) | (pack4<2>(s3.k) << 24);
+                    for (int u = 0; u < kEpBatch; ++u) {
+                        const int c = c0 + u * 32 + lane;
+                        v[u] = make_uint4(0, 0, 0, 0);
+                        if (c < cpr) v[u] = ld_stream_u4(src + c);
                     }
-                    if (sliced) reinterpret_cast<uint4*>(sliced)[c_row + c] = make_uint4(s0.k << sh, s1.k << sh, s2.k << sh, s3.k << sh);
-                    const uint32_t m = chunk_mask(s0, s1, s2, s3);
-                    mrow[c] = (uint16_t)m;
-                    cnt += __popc(m);
-                }
-            }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                    for (int u = 0; u < kEpBatch; ++u) {
+                        const int c = c0 + u * 32 + lane;
+                        if (c >= cpr) continue;
+                        const Sliced s0 = slice4(v[u].x, r), s1 = slice4(v[u].y, r), s2 = slice4(v[u].z, r), s3 = slice4(v[u].w, r);
+                        if (PACK_R == 4) {
+                            reinterpret_cast<uint2*>(packed)[c_row + c] =
+                                make_uint2(pack4<4>(s0.k) | (pack4<4>(s1.k) << 16), pack4<4>(s2.k) | (pack4<4>(s3.k) << 16));
+                        } else if (PACK_R == 2) {
+                            reinterpret_cast<uint32_t*>(packed)[c_row + c] =
+                                pack4<2>(s0.k) | (pack4<2>(s1.k) << 8) | (pack4<2>(s2.k) << 16) | (pack4<2>(s3.k) << 24);
+                        }
+                        if (sliced) reinterpret_cast<uint4*>(sliced)[c_row + c] = make_uint4(s0.k << sh, s1.k << sh, s2.k << sh, s3.k << sh);
+                        const uint32_t m = chunk_mask(s0, s1, s2, s3);
+                        mrow[c] = (uint16_t)m;
+                        cnt += __popc(m);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            }
+            if (lane == 0) row_off[lr] = cnt;
         }
-        if (lane == 0) row_cnt[warp] = cnt;
         __syncthreads();
         if (warp == 0) {
-            const int mine = lane < kEpRows ? row_cnt[lane] : 0;
-            int incl = mine;                                             // inclusive scan over the eight rows
+            uint32_t tile_total = 0;                                     // counts -> exclusive offsets, 32 rows at a time
+            for (int c0 = 0; c0 < T; c0 += 32) {
+                const int v = c0 + lane < T ? row_off[c0 + lane] : 0;
+                int incl = v;
 #pragma unroll
-            for (int o = 1; o < kEpRows; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += u;
+                }
+                if (c0 + lane < T) row_off[c0 + lane] = (int)tile_total + incl - v;
+                tile_total += (uint32_t)__shfl_sync(0xffffffffu, incl, 31);
             }
-            const uint32_t tile_total = (uint32_t)__shfl_sync(0xffffffffu, incl, kEpRows - 1);
-            const int64_t last_row = min(t * (int64_t)kEpRows + kEpRows - 1, N - 1);
+            const int64_t last_row = min(row0 + T - 1, N - 1);
             uint32_t base = 0;
             bool bad = false;
             if (t > 0) {
@@ -373,7 +386,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, ui
 #pragma unroll
                         for (int w = 0; w < kEpWindows; ++w) {
                             const int64_t j = look - 32 * w - lane;
-                            f[w] = j >= 0 ? ld_flag(row_ptr + j * kEpRows + kEpRows) : 0u;   // tiles before t are full
+                            f[w] = j >= 0 ? ld_flag(row_ptr + (j + 1) * T) : 0u;   // tiles before t are full
                             nothing |= f[w] == kEpNothing;
                         }
                         if (!__any_sync(0xffffffffu, nothing)) break;
@@ -396,17 +409,13 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, ui
                     look -= 32 * kEpWindows;
                 }
             }
-            if (bad) {
-                if (lane == 0) {
+            if (lane == 0) {
+                if (bad) {
                     st_flag(row_ptr + last_row + 1, kEpPoison);
                     report(dev_status, MATQ_ERR_TIMEOUT);
                     if (t == ntiles - 1) *total_out = 0;
-                }
-            } else {
-                const int64_t nrow = t * (int64_t)kEpRows + lane;
-                if (lane < kEpRows && nrow < last_row) row_ptr[nrow + 1] = base + (uint32_t)incl;
-                if (lane == 0) {                                         // the thread that wrote the partial replaces it
-                    st_flag(row_ptr + last_row + 1, base + tile_total);
+                } else {
+                    st_flag(row_ptr + last_row + 1, base + tile_total);   // the thread that wrote the partial replaces it
                     if (t == 0) row_ptr[0] = 0;
                     if (t == ntiles - 1) {
                         const int64_t total = (int64_t)base + tile_total;
@@ -414,68 +423,94 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, ui
                         if (total > capacity) report(dev_status, MATQ_ERR_CAPACITY);
                     }
                 }
+                base_s = base; total_s = tile_total; bad_s = bad ? 1 : 0;
             }
-            if (lane == 0) { tile_base_s = base; tile_bad_s = bad ? 1 : 0; }
         }
         __syncthreads();
-        if (n < N && cnt > 0 && !tile_bad_s) {
-            int64_t out = tile_base_s;
-            for (int w = 0; w < warp; ++w) out += row_cnt[w];
-            for (int c0 = 0; c0 < cpr; c0 += 8 * 32) {
-                uint32_t mask[8];
+        if (!bad_s) {
+            const int64_t last_row = min(row0 + T - 1, N - 1);
+            for (int i = 0; i < rows_per_warp; ++i) {
+                const int lr = i * nwarps + warp;
+                const int64_t n = row0 + lr;
+                if (n >= N) break;
+                const uint32_t excl = (uint32_t)row_off[lr];
+                const uint32_t cnt = (lr + 1 < T ? (uint32_t)row_off[lr + 1] : total_s) - excl;
+                if (lane == 0 && n < last_row) row_ptr[n + 1] = base_s + excl + cnt;
+                if (cnt == 0) continue;
+                const uint16_t* mrow = ep_mask + (size_t)lr * cpr;
+                int64_t out = (int64_t)base_s + excl;
+                for (int c0 = 0; c0 < cpr; c0 += 8 * 32) {
+                    uint32_t mask[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int c = c0 + j * 32 + lane;
-                    mask[j] = c < cpr ? mrow[c] : 0u;
-                }
-                uint32_t pk[3];                                   // inclusive lane scans, three 10-bit fields per word
-                pk[0] = __popc(mask[0]) | (__popc(mask[1]) << 10) | (__popc(mask[2]) << 20);
-                pk[1] = __popc(mask[3]) | (__popc(mask[4]) << 10) | (__popc(mask[5]) << 20);
-                pk[2] = __popc(mask[6]) | (__popc(mask[7]) << 10);
-                if (!__any_sync(0xffffffffu, (pk[0] | pk[1] | pk[2]) != 0)) continue;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-#pragma unroll
-                    for (int w = 0; w < 3; ++w) {
-                        const uint32_t v = __shfl_up_sync(0xffffffffu, pk[w], o);
-                        if (lane >= o) pk[w] += v;
+                    for (int j = 0; j < 8; ++j) {
+                        const int c = c0 + j * 32 + lane;
+                        mask[j] = c < cpr ? mrow[c] : 0u;
                     }
-                }
+                    uint32_t pk[3];                               // inclusive lane scans, three 10-bit fields per word
+                    pk[0] = __popc(mask[0]) | (__popc(mask[1]) << 10) | (__popc(mask[2]) << 20);
+                    pk[1] = __popc(mask[3]) | (__popc(mask[4]) << 10) | (__popc(mask[5]) << 20);
+                    pk[2] = __popc(mask[6]) | (__popc(mask[7]) << 10);
+                    if (!__any_sync(0xffffffffu, (pk[0] | pk[1] | pk[2]) != 0)) continue;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t incl = (pk[j / 3] >> (10 * (j % 3))) & 0x3ffu;
-                    const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-                    uint32_t m = mask[j];
-                    int64_t pos = out + incl - __popc(m);
-                    const int kb = (c0 + j * 32 + lane) * 16;
-                    while (m) {
-                        const int bpos = __ffs(m) - 1;
-                        if (pos < capacity) ovf_col[pos] = (uint16_t)(kb + bpos);
-                        ++pos;
-                        m &= m - 1;
+                    for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+                        for (int w = 0; w < 3; ++w) {
+                            const uint32_t v = __shfl_up_sync(0xffffffffu, pk[w], o);
+                            if (lane >= o) pk[w] += v;
+                        }
                     }
-                    out += tot;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t incl = (pk[j / 3] >> (10 * (j % 3))) & 0x3ffu;
+                        const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+                        uint32_t m = mask[j];
+                        int64_t pos = out + incl - __popc(m);
+                        const int kb = (c0 + j * 32 + lane) * 16;
+                        while (m) {
+                            const int bpos = __ffs(m) - 1;
+                            if (pos < capacity) ovf_col[pos] = (uint16_t)(kb + bpos);
+                            ++pos;
+                            m &= m - 1;
+                        }
+                        out += tot;
+                    }
                 }
             }
         }
-        __syncthreads();                                      // masks, counts and the base are reused by the next tile
+        __syncthreads();                                      // masks, offsets and the base are reused by the next tile
     }
 }
 
+// Returns MATQ_ERR_SHAPE when no tile fits the shared-memory budget (the caller then uses the three-kernel chain).
 template <int PACK_R>
 int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, uint8_t* sliced, int32_t* row_ptr,
               uint16_t* ovf_col, int64_t capacity, int64_t* total, int32_t* dev_status, cudaStream_t s) {
-    const size_t smem = (size_t)kEpRows * (size_t)(K / 16) * sizeof(uint16_t);
+    const int sms = sm_count();
+    const size_t row_smem = sizeof(int) + (size_t)(K / 16) * sizeof(uint16_t);
+    int nwarps = 32, rpw = 1;
+    for (;; nwarps >>= 1) {                                   // about one tile per SM, as many warps per tile as that allows
+        rpw = (int)((N + (int64_t)nwarps * sms - 1) / ((int64_t)nwarps * sms));
+        const int64_t rpw_fit = (int64_t)(kEpSmemLimit / (row_smem * nwarps));
+        if (rpw > rpw_fit) rpw = (int)rpw_fit;
+        if (nwarps == 8) break;
+        if (rpw >= 1 && (N + (int64_t)nwarps * rpw - 1) / ((int64_t)nwarps * rpw) >= (int64_t)sms * 85 / 100) break;
+    }
+    if (rpw < 1) return MATQ_ERR_SHAPE;
+    const int T = nwarps * rpw;
+    const size_t smem = (size_t)T * row_smem;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(slice_pack_ep<PACK_R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEpSmemLimit) != cudaSuccess)
+        return MATQ_ERR_CUDA;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_pack_ep<PACK_R>, kEpRows * 32, smem) != cudaSuccess ||
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_pack_ep<PACK_R>, nwarps * 32, smem) != cudaSuccess ||
         per_sm < 1)
         return MATQ_ERR_CUDA;
-    const int64_t ntiles = (N + kEpRows - 1) / kEpRows;
-    int64_t blocks = (int64_t)sm_count() * per_sm;            // all resident: the look-back waits rely on it
+    const int64_t ntiles = (N + T - 1) / T;
+    int64_t blocks = (int64_t)sms * per_sm;                   // all resident: the look-back waits rely on it
     if (blocks > ntiles) blocks = ntiles;
     if (cudaMemsetAsync(row_ptr, 0xff, (size_t)(N + 1) * sizeof(int32_t), s) != cudaSuccess) return MATQ_ERR_CUDA;
-    slice_pack_ep<PACK_R><<<(unsigned)blocks, kEpRows * 32, smem, s>>>(
-        q, N, (int)K, r, packed, sliced, reinterpret_cast<uint32_t*>(row_ptr), ovf_col, capacity, total, dev_status);
+    slice_pack_ep<PACK_R><<<(unsigned)blocks, nwarps * 32, smem, s>>>(
+        q, N, (int)K, r, rpw, packed, sliced, reinterpret_cast<uint32_t*>(row_ptr), ovf_col, capacity, total, dev_status);
     return launch_status();
 }
 
@@ -522,9 +557,11 @@ extern "C" int matq_slice_pack(const uint8_t* q, int64_t N, int64_t K, int c, in
     const bool vec = (K % 16 == 0) && aligned16(q) && (!packed || aligned16(packed)) &&
                      (!sliced_unpacked || aligned16(sliced_unpacked));
     if (want_ovf && vec && K <= 16384 && N * K < (int64_t(1) << 31)) {
-        if (!packed) return launch_ep<0>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
-        if (r == 4) return launch_ep<4>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
-        return launch_ep<2>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
+        int st;
+        if (!packed) st = launch_ep<0>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
+        else if (r == 4) st = launch_ep<4>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
+        else st = launch_ep<2>(q, N, K, r, packed, sliced_unpacked, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s);
+        if (st != MATQ_ERR_SHAPE) return st;
     }
     int32_t* row_count = nullptr;
     if (want_ovf) {
