@@ -41,22 +41,37 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else st5 = t5::launch<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         if (st5 != MATQ_ERR_SHAPE) return st5;     // a K too long for one cluster's shared memory falls through
     }
-    // Warp tile: 16*MT rows x K/SK.  Use two m-tiles per warp when there are plenty of rows (the staged activations
-    // are reused twice), then split K over as many warps as it takes to put about 16 warps on every SM.
+    // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at 24-32 warps per SM
+    // in a single wave of CTAs (measured optimum on B200 for 5-25 MB planes):
+    //   * few, long rows (at most one or two 16-row tiles per SM): one tile per CTA of 32 or 16 warps, SK = 32 / 16;
+    //   * otherwise CTAs of 8 warps, two m-tiles per warp when there are plenty of rows (r = 2 or a batch: the staged
+    //     activations are reused twice), and K split over up to 8 warps until about 16 warps sit on every SM.
     const int sms = sm_count();
-    const int mt = (N >= (int64_t)32 * 2 * sms) ? 2 : 1;
-    const int64_t tiles = (N + 16 * mt - 1) / (16 * mt);
     const int64_t n_qc = (K * r / 8 + 63) / 64;
-    int sk = 1;
-    while (sk < 8 && tiles * sk < (int64_t)16 * sms && n_qc / (2 * sk) >= 2) sk *= 2;
+    const int64_t tiles16 = (N + 15) / 16;
+    int mt = 1, sk = 1;
+    if (tiles16 <= sms && n_qc >= 32) sk = 32;
+    else if (tiles16 <= 2 * sms && n_qc >= 16) sk = 16;
+    else {
+        mt = (N >= (int64_t)64 * sms || (N >= (int64_t)48 * sms && (r == 2 || B > 1))) ? 2 : 1;
+        const int64_t tiles = (N + 16 * mt - 1) / (16 * mt);
+        while (sk < 8 && tiles * sk < (int64_t)16 * sms && n_qc / (2 * sk) >= 1) sk *= 2;
+    }
     int st;
 #define MATQ_GEMV_T(RR, MT, NT, SK) launch_gemv_tensor<RR, MT, NT, SK>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+#define MATQ_GEMV_W(RR, NT, W) launch_gemv_tensor<RR, 1, NT, W, W>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
 #define MATQ_GEMV_S(RR, MT, NT) ((sk == 8) ? MATQ_GEMV_T(RR, MT, NT, 8) : (sk == 4) ? MATQ_GEMV_T(RR, MT, NT, 4) : (sk == 2) ? MATQ_GEMV_T(RR, MT, NT, 2) : MATQ_GEMV_T(RR, MT, NT, 1))
 #define MATQ_GEMV_R(MT, NT) ((r == 8) ? MATQ_GEMV_S(8, MT, NT) : (r == 4) ? MATQ_GEMV_S(4, MT, NT) : MATQ_GEMV_S(2, MT, NT))
-    if (B <= 8) st = (mt == 2) ? MATQ_GEMV_R(2, 1) : MATQ_GEMV_R(1, 1);
+#define MATQ_GEMV_RW(NT, W) ((r == 8) ? MATQ_GEMV_W(8, NT, W) : (r == 4) ? MATQ_GEMV_W(4, NT, W) : MATQ_GEMV_W(2, NT, W))
+    if (sk >= 16) {                // few, long rows: one 16-row tile per CTA, K split over 16 or 32 warps
+        if (B <= 8) st = (sk == 32) ? MATQ_GEMV_RW(1, 32) : MATQ_GEMV_RW(1, 16);
+        else st = (sk == 32) ? MATQ_GEMV_RW(2, 32) : MATQ_GEMV_RW(2, 16);
+    } else if (B <= 8) st = (mt == 2) ? MATQ_GEMV_R(2, 1) : MATQ_GEMV_R(1, 1);
     else st = (mt == 2) ? MATQ_GEMV_R(2, 2) : MATQ_GEMV_R(1, 2);
+#undef MATQ_GEMV_RW
 #undef MATQ_GEMV_R
 #undef MATQ_GEMV_S
+#undef MATQ_GEMV_W
 #undef MATQ_GEMV_T
     if (st == MATQ_ERR_SHAPE) {   // the staged activations of this call do not fit in shared memory: FMA path
         if (r == 8) launch_gemv_cuda_core<8>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);

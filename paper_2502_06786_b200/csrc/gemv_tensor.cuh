@@ -41,8 +41,6 @@
 
 namespace matq {
 
-constexpr int kGemvThreads = 256;
-constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kGemvDepth = 3;               // chunks requested ahead of the one being multiplied
 
 struct GemvTensorParams {
@@ -57,8 +55,9 @@ struct GemvTensorParams {
     int64_t row_bytes;
     int B;            // batch columns in use
     int bpad;         // batch columns staged: 1, 2, 4, 8 or 16
+    int bpad_log2;
     int n_qc;         // 64-byte chunks per row (last one may be partial)
-    int qc_per_warp;  // chunks per K slice
+    int qc_pass;      // chunks whose activations are staged at a time (a multiple of nothing in particular; >= 1)
     int pdl;
 };
 
@@ -144,9 +143,10 @@ __device__ __forceinline__ void stage_word(const __nv_bfloat16* xw, uint4* dst, 
     }
 }
 
-template <int R, int MT, int NT, int SK>
-__global__ void __launch_bounds__(kGemvThreads)
+template <int R, int MT, int NT, int SK, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, (MT == 1 ? 32 : 16) / WARPS)   // MT = 1: 64 registers, a full SM of warps
 gemv_tensor(const GemvTensorParams P) {
+    constexpr int kGemvThreads = WARPS * 32, kGemvWarps = WARPS;
     using Fmt = GemvFmt<R>;
     constexpr int kTileRows = 16 * MT;                    // rows of a warp
     constexpr int kTiles = kGemvWarps / SK;               // row tiles of a CTA
@@ -164,13 +164,21 @@ gemv_tensor(const GemvTensorParams P) {
     const int g = lane >> 2, t = lane & 3;
     const int tile = warp / SK, ks = warp % SK;
     const int64_t row0 = (int64_t)blockIdx.x * kRows + (int64_t)tile * kTileRows;
-    const int q_lo = ks * P.qc_per_warp;
-    const int q_hi = min(q_lo + P.qc_per_warp, P.n_qc);
+    // K is walked in passes of qc_pass chunks (one pass unless the staged activations would not fit in shared memory);
+    // inside a pass the SK warps of a row tile take consecutive slices of its chunks.
+    int pass_lo = 0, pass_hi = min(P.qc_pass, P.n_qc);
+    int q_lo, q_hi;
+    auto set_slice = [&]() {
+        const int per_warp = (pass_hi - pass_lo + SK - 1) / SK;
+        q_lo = pass_lo + ks * per_warp;
+        q_hi = min(q_lo + per_warp, pass_hi);
+    };
+    set_slice();
     const int bpad = P.bpad;
 
     // shared memory: x' fragments for all of K | partial tiles [warp][kTileRows][kMaxB] (SK > 1 only)
     uint4* xs = reinterpret_cast<uint4*>(smem_raw);
-    float* part = reinterpret_cast<float*>(smem_raw + (size_t)P.n_qc * 4 * kPG * bpad * 64);
+    float* part = reinterpret_cast<float*>(smem_raw + (size_t)min(P.qc_pass, P.n_qc) * 4 * kPG * bpad * 64);
 
     // ---- weights of the first chunks are requested before anything that depends on the previous kernel
     const uint8_t* wrow[2 * MT];
@@ -207,39 +215,6 @@ gemv_tensor(const GemvTensorParams P) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
 
-    // ---- stage x' (pre-scaled activations in B-fragment order) and the two sums per batch column.
-    // Item i = ((q*4 + j) * bpad + gg) * 4 + tt covers one packed word's worth of activations.  (i >> 2) % bpad
-    // is the batch column and 256 / 4 is a multiple of bpad, so every group of 4 lanes sees a single column.
-    {
-        const int items = P.n_qc * 4 * bpad * 4;
-        float sx = 0.f, sxp = 0.f;
-        for (int i = tid; i < items; i += kGemvThreads) {
-            const int tt = i & 3;
-            const int gg = (i >> 2) % bpad;
-            const int qj = (i >> 2) / bpad;              // q*4 + j
-            const int64_t kb = (int64_t)(qj >> 2) * kWq + tt * (kWq / 4) + (qj & 3) * Fmt::kWeightsPerWord;
-            uint4* dst = xs + ((size_t)qj * kPG * bpad + gg) * 4 + tt;
-            if (gg < P.B && kb < P.K) {                   // K % 128 == 0: a word lies inside or outside
-                stage_word<R>(P.x + (int64_t)gg * P.ldx + kb, dst, bpad * 4, sx, sxp);
-            } else {
-                dst[0] = make_uint4(0, 0, 0, 0);
-                if (kPG == 2) dst[bpad * 4] = make_uint4(0, 0, 0, 0);
-            }
-        }
-        sx += __shfl_xor_sync(0xffffffffu, sx, 1);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 1);
-        sx += __shfl_xor_sync(0xffffffffu, sx, 2);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 2);
-        if (t == 0) { s_grp[0][tid >> 2] = sx; s_grp[1][tid >> 2] = sxp; }
-    }
-    __syncthreads();
-    if (tid < kMaxB) {
-        float sx = 0.f, sxp = 0.f;
-        if (tid < bpad)
-            for (int h = tid; h < kGemvThreads / 4; h += bpad) { sx += s_grp[0][h]; sxp += s_grp[1][h]; }
-        s_sumx[tid] = sx;          // read after the barrier that precedes the epilogue
-        s_sumxp[tid] = sxp;
-    }
-
-    // ---- main loop over this warp's chunks
     float acc[kSets][MT][NT][4];
 #pragma unroll
     for (int c = 0; c < kSets; ++c)
@@ -250,39 +225,79 @@ gemv_tensor(const GemvTensorParams P) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[c][mt][nt][i] = 0.f;
 
-    for (int q0 = q_lo; q0 < q_hi; q0 += kGemvDepth) {
+    float sx = 0.f, sxp = 0.f;                            // this thread's share of sum(x) and sum(x') of its column
+    for (;;) {
+        // ---- stage x' (pre-scaled activations in B-fragment order) of this pass and add to the two sums.
+        // Item i = ((q*4 + j) * bpad + gg) * 4 + tt covers one packed word's worth of activations.  (i >> 2) % bpad
+        // is the batch column and threads / 4 is a multiple of bpad, so every group of 4 lanes sees a single column.
+        {
+            const int items = (pass_hi - pass_lo) * 4 * bpad * 4;
+            const int qj0 = pass_lo * 4;
+            for (int i = tid; i < items; i += kGemvThreads) {
+                const int tt = i & 3;
+                const int gg = (i >> 2) & (bpad - 1);        // bpad is a power of two
+                const int qjl = (i >> 2) >> P.bpad_log2;     // (q - pass_lo)*4 + j
+                const int qj = qj0 + qjl;
+                const int64_t kb = (int64_t)(qj >> 2) * kWq + tt * (kWq / 4) + (qj & 3) * Fmt::kWeightsPerWord;
+                uint4* dst = xs + ((size_t)qjl * kPG * bpad + gg) * 4 + tt;
+                if (gg < P.B && kb < P.K) {                   // K % 128 == 0: a word lies inside or outside
+                    stage_word<R>(P.x + (int64_t)gg * P.ldx + kb, dst, bpad * 4, sx, sxp);
+                } else {
+                    dst[0] = make_uint4(0, 0, 0, 0);
+                    if (kPG == 2) dst[bpad * 4] = make_uint4(0, 0, 0, 0);
+                }
+            }
+        }
+        const bool last_pass = pass_hi >= P.n_qc;            // uniform over the CTA
+        if (last_pass) {
+            sx += __shfl_xor_sync(0xffffffffu, sx, 1);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 1);
+            sx += __shfl_xor_sync(0xffffffffu, sx, 2);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 2);
+            if (t == 0) { s_grp[0][tid >> 2] = sx; s_grp[1][tid >> 2] = sxp; }
+        }
+        __syncthreads();
+        if (last_pass && tid < kMaxB) {
+            float tx = 0.f, txp = 0.f;
+            if (tid < bpad)
+                for (int h = tid; h < kGemvThreads / 4; h += bpad) { tx += s_grp[0][h]; txp += s_grp[1][h]; }
+            s_sumx[tid] = tx;          // read after the barrier that precedes the epilogue
+            s_sumxp[tid] = txp;
+        }
+
+        // ---- this warp's chunks of the pass
+        for (int q0 = q_lo; q0 < q_hi; q0 += kGemvDepth) {
 #pragma unroll
-        for (int d = 0; d < kGemvDepth; ++d) {
-            const int q = q0 + d;
-            if (q < q_hi) {                               // warp-uniform
-                uint4 wv[2 * MT];
+            for (int d = 0; d < kGemvDepth; ++d) {
+                const int q = q0 + d;
+                if (q < q_hi) {                               // warp-uniform
+                    uint4 wv[2 * MT];
 #pragma unroll
-                for (int h = 0; h < 2 * MT; ++h) wv[h] = wbuf[d][h];
-                load_chunk(q + kGemvDepth, wbuf[d]);
+                    for (int h = 0; h < 2 * MT; ++h) wv[h] = wbuf[d][h];
+                    load_chunk(q + kGemvDepth, wbuf[d]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                    for (int j = 0; j < 4; ++j) {
 #pragma unroll
-                    for (int pg = 0; pg < kPG; ++pg) {
-                        uint4 xb[NT];
+                        for (int pg = 0; pg < kPG; ++pg) {
+                            uint4 xb[NT];
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            xb[nt] = make_uint4(0, 0, 0, 0);
-                            const int gb = g + 8 * nt;
-                            if (gb < bpad) xb[nt] = xs[(((size_t)q * 4 + j) * kPG + pg) * bpad * 4 + gb * 4 + t];
-                        }
+                            for (int nt = 0; nt < NT; ++nt) {
+                                xb[nt] = make_uint4(0, 0, 0, 0);
+                                const int gb = g + 8 * nt;
+                                if (gb < bpad) xb[nt] = xs[(((size_t)(q - pass_lo) * 4 + j) * kPG + pg) * bpad * 4 + gb * 4 + t];
+                            }
 #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int p = pg * 4 + 2 * u;
+                            for (int u = 0; u < 2; ++u) {
+                                const int p = pg * 4 + 2 * u;
 #pragma unroll
-                            for (int mt = 0; mt < MT; ++mt) {
-                                const uint32_t w_lo = (j == 0 ? wv[2 * mt].x : j == 1 ? wv[2 * mt].y : j == 2 ? wv[2 * mt].z : wv[2 * mt].w);
-                                const uint32_t w_hi = (j == 0 ? wv[2 * mt + 1].x : j == 1 ? wv[2 * mt + 1].y : j == 2 ? wv[2 * mt + 1].z : wv[2 * mt + 1].w);
-                                const uint32_t a0 = field_pair<R>(w_lo, p), a1 = field_pair<R>(w_hi, p);
-                                const uint32_t a2 = field_pair<R>(w_lo, p + 1), a3 = field_pair<R>(w_hi, p + 1);
+                                for (int mt = 0; mt < MT; ++mt) {
+                                    const uint32_t w_lo = (j == 0 ? wv[2 * mt].x : j == 1 ? wv[2 * mt].y : j == 2 ? wv[2 * mt].z : wv[2 * mt].w);
+                                    const uint32_t w_hi = (j == 0 ? wv[2 * mt + 1].x : j == 1 ? wv[2 * mt + 1].y : j == 2 ? wv[2 * mt + 1].z : wv[2 * mt + 1].w);
+                                    const uint32_t a0 = field_pair<R>(w_lo, p), a1 = field_pair<R>(w_hi, p);
+                                    const uint32_t a2 = field_pair<R>(w_lo, p + 1), a3 = field_pair<R>(w_hi, p + 1);
 #pragma unroll
-                                for (int nt = 0; nt < NT; ++nt) {
-                                    const uint32_t b0 = u ? xb[nt].z : xb[nt].x, b1 = u ? xb[nt].w : xb[nt].y;
-                                    mma_bf16_16816(acc[u % kSets][mt][nt], a0, a1, a2, a3, b0, b1);
+                                    for (int nt = 0; nt < NT; ++nt) {
+                                        const uint32_t b0 = u ? xb[nt].z : xb[nt].x, b1 = u ? xb[nt].w : xb[nt].y;
+                                        mma_bf16_16816(acc[u % kSets][mt][nt], a0, a1, a2, a3, b0, b1);
+                                    }
                                 }
                             }
                         }
@@ -290,6 +305,14 @@ gemv_tensor(const GemvTensorParams P) {
                 }
             }
         }
+        if (last_pass) break;
+        // ---- next pass: request its first chunks, then wait until every warp is done with the staged activations
+        pass_lo = pass_hi;
+        pass_hi = min(pass_lo + P.qc_pass, P.n_qc);
+        set_slice();
+#pragma unroll
+        for (int d = 0; d < kGemvDepth; ++d) load_chunk(q_lo + d, wbuf[d]);
+        __syncthreads();
     }
     if (kSets == 2) {
 #pragma unroll
@@ -349,11 +372,12 @@ gemv_tensor(const GemvTensorParams P) {
 }
 
 // Host side: geometry and launch.
-template <int R, int MT, int NT, int SK>
+template <int R, int MT, int NT, int SK, int WARPS = 8>
 inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const float* alpha, const float* zero,
                               const int32_t* ovf_row_ptr, const uint16_t* ovf_col, const void* x, int B, int64_t ldx,
                               float* y, int64_t ldy, bool pdl, cudaStream_t s) {
     using Fmt = GemvFmt<R>;
+    constexpr int kGemvThreads = WARPS * 32, kGemvWarps = WARPS;
     constexpr int kRows = 16 * MT * (kGemvWarps / SK), kMaxB = 8 * NT;
     constexpr int kPG = Fmt::kPairs / 4;
     GemvTensorParams P;
@@ -364,11 +388,17 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     P.B = B;
     P.bpad = B <= 1 ? 1 : B <= 2 ? 2 : B <= 4 ? 4 : B <= 8 ? 8 : 16;
     P.n_qc = (int)((P.row_bytes + 63) / 64);
-    P.qc_per_warp = (P.n_qc + SK - 1) / SK;
     P.pdl = pdl ? 1 : 0;
-    const size_t smem = (size_t)P.n_qc * 4 * kPG * P.bpad * 64 + (SK > 1 ? (size_t)kGemvWarps * 16 * MT * kMaxB * sizeof(float) : 0);
-    if (smem > 200 * 1024) return MATQ_ERR_SHAPE;          // activations of one call must fit in shared memory
-    auto kern = gemv_tensor<R, MT, NT, SK>;
+    P.bpad_log2 = P.bpad == 1 ? 0 : P.bpad == 2 ? 1 : P.bpad == 4 ? 2 : P.bpad == 8 ? 3 : 4;
+    // Shared memory: the staged activations of one pass (64 * 4 * kPG * bpad bytes per chunk) + the split-K partials.
+    // Passes are as long as ~150 KB allow (one pass for all decode shapes up to K = 9216 at B = 8).
+    const size_t part_bytes = SK > 1 ? (size_t)kGemvWarps * 16 * MT * kMaxB * sizeof(float) : 0;
+    const size_t chunk_bytes = (size_t)4 * kPG * P.bpad * 64;
+    const int fit = (int)((150 * 1024 - part_bytes) / chunk_bytes);
+    const int passes = (P.n_qc + fit - 1) / fit;
+    P.qc_pass = (P.n_qc + passes - 1) / passes;
+    const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
+    auto kern = gemv_tensor<R, MT, NT, SK, WARPS>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
