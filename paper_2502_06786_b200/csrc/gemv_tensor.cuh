@@ -30,7 +30,9 @@
 // still computing, only the activations depend on it.  With SK = 1 a warp
 // finishes its outputs alone and writes y from its accumulators; with SK > 1
 // the SK warps of a row tile are summed through shared memory in a fixed
-// order.  No global scratch, no atomics: results are deterministic.
+// order.  No global scratch, no atomics: results are deterministic.  The
+// extra-precision overflow lists are walked by a few threads per row in
+// parallel with the staging of the activations.
 //
 // The activations are staged once per CTA into shared memory as x' in exactly
 // the order the B fragments are consumed, so a thread fetches the B registers
@@ -143,7 +145,7 @@ __device__ __forceinline__ void stage_word(const __nv_bfloat16* xw, uint4* dst, 
     }
 }
 
-template <int R, int MT, int NT, int SK, int WARPS>
+template <int R, int MT, int NT, int SK, int WARPS, bool EP>
 __global__ void __launch_bounds__(WARPS * 32, (MT == 1 ? 32 : 16) / WARPS)   // MT = 1: 64 registers, a full SM of warps
 gemv_tensor(const GemvTensorParams P) {
     constexpr int kGemvThreads = WARPS * 32, kGemvWarps = WARPS;
@@ -159,6 +161,9 @@ gemv_tensor(const GemvTensorParams P) {
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ float s_sumx[kMaxB], s_sumxp[kMaxB], s_grp[2][kGemvThreads / 4];
+    __shared__ float s_ep[EP ? kRows : 1][kMaxB];         // extra-precision correction per row and batch column
+    constexpr int kRowThreads = kGemvThreads / kRows;     // = 2 SK / MT consecutive threads per row of the CTA
+    constexpr int kTPR = kRowThreads > 32 ? 32 : kRowThreads;   // of which this many walk the row's overflow list
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -210,10 +215,29 @@ gemv_tensor(const GemvTensorParams P) {
         z_pre[h] = wok[h] ? P.zero[row] : 0.f;
     }
 
+    // Extra precision (Errata, Eq. 8): an overflow column's field is one higher than the stored, clamped one, so its
+    // activation is added once more.  kTPR threads share a row's list; the list (weights-side data) is read before
+    // the dependency wait, the activations it points at right after it, and the sums land in s_ep before the
+    // barrier that precedes the epilogue.
+    const int ep_row = tid / kRowThreads, ep_j = tid % kRowThreads;
+    int ep_p = 0, ep_hi = 0, ep_c0 = 0;
+    if (EP && ep_j < kTPR) {
+        const int64_t row = (int64_t)blockIdx.x * kRows + ep_row;
+        if (row < P.N) {
+            ep_p = P.ovf_row_ptr[row] + ep_j;
+            ep_hi = P.ovf_row_ptr[row + 1];
+            if (ep_p < ep_hi) ep_c0 = P.ovf_col[ep_p];
+        }
+    }
+
     if (P.pdl) {
         asm volatile("griddepcontrol.launch_dependents;");
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
+
+    // activation (batch column 0) of this thread's first overflow column: requested now, used after the staging
+    float ep_x0 = 0.f;
+    if (EP && ep_p < ep_hi) ep_x0 = __bfloat162float(P.x[ep_c0]);
 
     float acc[kSets][MT][NT][4];
 #pragma unroll
@@ -246,6 +270,23 @@ gemv_tensor(const GemvTensorParams P) {
                     dst[0] = make_uint4(0, 0, 0, 0);
                     if (kPG == 2) dst[bpad * 4] = make_uint4(0, 0, 0, 0);
                 }
+            }
+        }
+        if (EP && pass_lo == 0) {                             // uniform over the CTA
+            for (int b = 0; b < P.B; ++b) {
+                const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
+                float ev = b == 0 ? ep_x0 : (ep_p < ep_hi ? __bfloat162float(xr[ep_c0]) : 0.f);
+                for (int p = ep_p + kTPR; p < ep_hi; p += 4 * kTPR) {      // lists longer than kTPR entries
+                    int col[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) col[u] = p + u * kTPR < ep_hi ? (int)P.ovf_col[p + u * kTPR] : -1;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (col[u] >= 0) ev += __bfloat162float(xr[col[u]]);
+                }
+#pragma unroll
+                for (int o = kTPR / 2; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
+                if (ep_j == 0) s_ep[ep_row][b] = ev;
             }
         }
         const bool last_pass = pass_hi >= P.n_qc;            // uniform over the CTA
@@ -360,13 +401,7 @@ gemv_tensor(const GemvTensorParams P) {
                 const int64_t row = row0 + mt * 16 + g + (i >> 1) * 8;
                 if (!wok[h] || b >= P.B) continue;
                 float v = acc[0][mt][nt][i] - 128.0f * s_sumxp[b];
-                if (P.ovf_row_ptr) {                       // extra-precision columns: their field is one higher
-                    const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
-                    const int32_t pe = P.ovf_row_ptr[row + 1];
-                    float ev = 0.f;
-                    for (int32_t p = P.ovf_row_ptr[row]; p < pe; ++p) ev += __bfloat162float(xr[P.ovf_col[p]]);
-                    v += ev;
-                }
+                if (EP) v += s_ep[tile * kTileRows + mt * 16 + g + (i >> 1) * 8][b];
                 P.y[(int64_t)b * P.ldy + row] = a_pre[h] * (v * (float)(1 << sh) - z_pre[h] * s_sumx[b]);
             }
 }
@@ -398,7 +433,7 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     const int passes = (P.n_qc + fit - 1) / fit;
     P.qc_pass = (P.n_qc + passes - 1) / passes;
     const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
-    auto kern = gemv_tensor<R, MT, NT, SK, WARPS>;
+    auto kern = ovf_row_ptr ? gemv_tensor<R, MT, NT, SK, WARPS, true> : gemv_tensor<R, MT, NT, SK, WARPS, false>;
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
