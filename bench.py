@@ -44,6 +44,12 @@ if ROOT not in sys.path:
 from paper_2502_06786_b200 import synth  # noqa: E402
 
 METRIC = "sliced int{8,4,2} GEMV HBM GB/s (% of peak); multi-precision GEMM TFLOP/s"
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised under
+# profiles/, for kernels that have not changed since; a stage that is missing here reports traffic = null.
+NCU_TRAFFIC = {"quantize": 42750000}
+NCU_TRAFFIC_NOTE = {"quantize": "ncu, one 9216x2304 launch: 42.49 MB read (= the algorithmic 42.47 MB) + 0.26 MB written; "
+                                "the 21.2 MB of codes were still in the L2 when the launch ended, so the write-back "
+                                "shows up in later launches"}
 CONFIG_ID = 2
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -336,9 +342,11 @@ def run_cuda(args, rank, world, local_rank):
     else:
         ach = nbytes / (stage_ms[dom] * 1e-3) / 1e9
         roofline = dict(kernel=name, bound="hbm", achieved=round(ach, 1), peak=peaks["hbm_gbs"], unit="GB/s",
-                        frac=round(ach / peaks["hbm_gbs"], 4), traffic=None, peak_source=peaks["source"],
+                        frac=round(ach / peaks["hbm_gbs"], 4), traffic=NCU_TRAFFIC.get(name), peak_source=peaks["source"],
                         avg_launch_us=round(stage_ms[dom] * 1e3 / len(shapes), 3),
                         bytes_per_launch=nbytes // len(shapes))
+        if name in NCU_TRAFFIC_NOTE:
+            roofline["traffic_note"] = NCU_TRAFFIC_NOTE[name]
 
     gpu_launches = sum((p[2] if p[2] is not None else 2 * len(shapes)) for p in plan)
 
