@@ -301,6 +301,13 @@ __device__ __forceinline__ uint32_t chunk_mask(const Sliced& s0, const Sliced& s
            (gather_byte_lsbs(s3.ov) << 12);
 }
 
+// Sets every flag word to "nothing yet".  The one-pass kernel is launched as its programmatic dependent: it slices,
+// packs and counts while this runs and only waits for it before it touches the first flag.
+__global__ void __launch_bounds__(256) ep_init_flags(uint32_t* __restrict__ row_ptr, int64_t n) {
+    asm volatile("griddepcontrol.launch_dependents;");
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) row_ptr[i] = kEpNothing;
+}
+
 template <int PACK_R>
 __global__ void __launch_bounds__(1024)
 slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, int rows_per_warp,
@@ -358,6 +365,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
             }
             if (lane == 0) row_off[lr] = cnt;
         }
+        if (t == (int64_t)blockIdx.x) asm volatile("griddepcontrol.wait;" ::: "memory");   // the flags are initialised
         __syncthreads();
         if (warp == 0) {
             uint32_t tile_total = 0;                                     // counts -> exclusive offsets, 32 rows at a time
@@ -508,9 +516,25 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     const int64_t ntiles = (N + T - 1) / T;
     int64_t blocks = (int64_t)sms * per_sm;                   // all resident: the look-back waits rely on it
     if (blocks > ntiles) blocks = ntiles;
-    if (cudaMemsetAsync(row_ptr, 0xff, (size_t)(N + 1) * sizeof(int32_t), s) != cudaSuccess) return MATQ_ERR_CUDA;
-    slice_pack_ep<PACK_R><<<(unsigned)blocks, nwarps * 32, smem, s>>>(
-        q, N, (int)K, r, rpw, packed, sliced, reinterpret_cast<uint32_t*>(row_ptr), ovf_col, capacity, total, dev_status);
+    const int64_t init_blocks = (N + 1 + 255) / 256;
+    ep_init_flags<<<(unsigned)(init_blocks < 2 * sms ? init_blocks : 2 * sms), 256, 0, s>>>(reinterpret_cast<uint32_t*>(row_ptr), N + 1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3((unsigned)(nwarps * 32));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int K32 = (int)K;
+    uint32_t* flags = reinterpret_cast<uint32_t*>(row_ptr);
+    if (cudaLaunchKernelEx(&cfg, slice_pack_ep<PACK_R>, q, N, K32, r, rpw, packed, sliced, flags, ovf_col, capacity, total,
+                           dev_status) != cudaSuccess) {
+        cudaGetLastError();
+        return MATQ_ERR_CUDA;
+    }
     return launch_status();
 }
 
