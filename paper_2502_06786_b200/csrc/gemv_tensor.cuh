@@ -296,12 +296,19 @@ gemv_tensor(const GemvTensorParams P) {
             if (t == 0) { s_grp[0][tid >> 2] = sx; s_grp[1][tid >> 2] = sxp; }
         }
         __syncthreads();
-        if (last_pass && tid < kMaxB) {
+        if (last_pass && warp == 0) {
+            // entry h of s_grp belongs to batch column h % bpad (bpad divides 32): lanes congruent modulo bpad are summed
             float tx = 0.f, txp = 0.f;
-            if (tid < bpad)
-                for (int h = tid; h < kGemvThreads / 4; h += bpad) { tx += s_grp[0][h]; txp += s_grp[1][h]; }
-            s_sumx[tid] = tx;          // read after the barrier that precedes the epilogue
-            s_sumxp[tid] = txp;
+#pragma unroll
+            for (int h = 0; h < kGemvThreads / 4; h += 32) { tx += s_grp[0][h + lane]; txp += s_grp[1][h + lane]; }
+            for (int o = 16; o >= bpad; o >>= 1) {
+                tx += __shfl_xor_sync(0xffffffffu, tx, o);
+                txp += __shfl_xor_sync(0xffffffffu, txp, o);
+            }
+            if (lane < kMaxB) {        // read after the barrier that precedes the epilogue
+                s_sumx[lane] = lane < bpad ? tx : 0.f;
+                s_sumxp[lane] = lane < bpad ? txp : 0.f;
+            }
         }
 
         // ---- this warp's chunks of the pass
