@@ -162,6 +162,7 @@ gemv_tensor(const GemvTensorParams P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ float s_sumx[kMaxB], s_sumxp[kMaxB], s_grp[2][kGemvThreads / 4];
     __shared__ float s_ep[EP ? kRows : 1][kMaxB];         // extra-precision correction per row and batch column
+    __shared__ float s_alpha[SK > 1 ? kRows : 1], s_zero[SK > 1 ? kRows : 1];
     constexpr int kRowThreads = kGemvThreads / kRows;     // = 2 SK / MT consecutive threads per row of the CTA
     constexpr int kTPR = kRowThreads > 32 ? 32 : kRowThreads;   // of which this many walk the row's overflow list
 
@@ -206,13 +207,22 @@ gemv_tensor(const GemvTensorParams P) {
 #pragma unroll
     for (int d = 0; d < kGemvDepth; ++d) load_chunk(q_lo + d, wbuf[d]);
 
-    // scale and zero point of the rows this thread finishes (rows g and g+8 of every m-tile)
+    // scale and zero point: with SK = 1 a thread finishes rows g and g+8 of every m-tile from its accumulators and
+    // keeps them in registers; with SK > 1 the CTA's rows are parked in shared memory for the shared epilogue.
     float a_pre[2 * MT], z_pre[2 * MT];
+    if (SK == 1) {
 #pragma unroll
-    for (int h = 0; h < 2 * MT; ++h) {
-        const int64_t row = row0 + (h >> 1) * 16 + (h & 1) * 8 + g;
-        a_pre[h] = wok[h] ? P.alpha[row] : 0.f;
-        z_pre[h] = wok[h] ? P.zero[row] : 0.f;
+        for (int h = 0; h < 2 * MT; ++h) {
+            const int64_t row = row0 + (h >> 1) * 16 + (h & 1) * 8 + g;
+            a_pre[h] = wok[h] ? P.alpha[row] : 0.f;
+            z_pre[h] = wok[h] ? P.zero[row] : 0.f;
+        }
+    } else {
+        for (int rl = tid; rl < kRows; rl += kGemvThreads) {
+            const int64_t row = (int64_t)blockIdx.x * kRows + rl;
+            s_alpha[rl] = row < P.N ? P.alpha[row] : 0.f;
+            s_zero[rl] = row < P.N ? P.zero[row] : 0.f;
+        }
     }
 
     // Extra precision (Errata, Eq. 8): an overflow column's field is one higher than the stored, clamped one, so its
@@ -384,18 +394,21 @@ gemv_tensor(const GemvTensorParams P) {
     }
     __syncthreads();                                      // publishes s_sumx / s_sumxp and the partial tiles
     if (SK > 1) {
-        if (ks != 0) return;
-        const float* base = part + (size_t)(tile * SK) * kTileRows * kMaxB;
+        // Every thread finishes outputs: output o = (row of the CTA) * kMaxB + batch column sums its SK partials in
+        // a fixed order and is scaled with the row's alpha / zero (parked in shared memory at the start).
+        for (int o = tid; o < kRows * kMaxB; o += kGemvThreads) {
+            const int b = o % kMaxB, row_l = o / kMaxB;
+            const int64_t row = (int64_t)blockIdx.x * kRows + row_l;
+            if (b >= P.B || row >= P.N) continue;
+            const float* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kMaxB + b;
+            float v = src[0];
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int off = (mt * 16 + g + (i >> 1) * 8) * kMaxB + nt * 8 + 2 * t + (i & 1);
-#pragma unroll
-                    for (int s = 1; s < SK; ++s) acc[0][mt][nt][i] += base[(size_t)s * kTileRows * kMaxB + off];
-                }
+            for (int sidx = 1; sidx < SK; ++sidx) v += src[(size_t)sidx * kTileRows * kMaxB];
+            v -= 128.0f * s_sumxp[b];
+            if (EP) v += s_ep[row_l][b];
+            P.y[(int64_t)b * P.ldy + row] = s_alpha[row_l] * (v * (float)(1 << sh) - s_zero[row_l] * s_sumx[b]);
+        }
+        return;
     }
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
