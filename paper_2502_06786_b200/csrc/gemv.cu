@@ -41,21 +41,26 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else st5 = t5::launch<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         if (st5 != MATQ_ERR_SHAPE) return st5;     // a K too long for one cluster's shared memory falls through
     }
-    // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at 24-32 warps per SM
-    // in a single wave of CTAs (measured optimum on B200 for 5-25 MB planes):
+    // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at ONE wave of CTAs
+    // (a second, partly filled wave costs up to 40 %; measured on B200 for 4-26 MB planes):
     //   * few, long rows (at most one or two 16-row tiles per SM): one tile per CTA of 32 or 16 warps, SK = 32 / 16;
-    //   * otherwise CTAs of 8 warps, two m-tiles per warp when there are plenty of rows (r = 2 or a batch: the staged
-    //     activations are reused twice), and K split over up to 8 warps until about 16 warps sit on every SM.
+    //   * otherwise CTAs of 8 warps with two m-tiles per warp (the staged activations are reused twice; two such
+    //     CTAs fit an SM) and the finest K split (8, else 4) that still fits one wave; if neither does, SK = 8 and
+    //     several waves.
     const int sms = sm_count();
     const int64_t n_qc = (K * r / 8 + 63) / 64;
     const int64_t tiles16 = (N + 15) / 16;
     int mt = 1, sk = 1;
-    if (tiles16 <= sms && n_qc >= 32) sk = 32;
-    else if (tiles16 <= 2 * sms && n_qc >= 16) sk = 16;
-    else {
-        mt = (N >= (int64_t)64 * sms || (N >= (int64_t)48 * sms && (r == 2 || B > 1))) ? 2 : 1;
-        const int64_t tiles = (N + 16 * mt - 1) / (16 * mt);
-        while (sk < 8 && tiles * sk < (int64_t)16 * sms && n_qc / (2 * sk) >= 1) sk *= 2;
+    if (tiles16 <= sms && n_qc >= 16) sk = 32;
+    else if (tiles16 <= 2 * sms && n_qc >= 8) sk = 16;
+    else if (tiles16 <= 2 * sms) {                       // few short rows: as many warps as there are chunks
+        while (sk < 8 && n_qc / (2 * sk) >= 1) sk *= 2;
+    } else {
+        mt = 2;
+        const int64_t tiles32 = (N + 31) / 32;
+        sk = 8;
+        if (tiles32 > 2 * sms && (tiles32 + 1) / 2 <= 2 * sms && n_qc >= 4) sk = 4;
+        while (sk > 1 && n_qc < sk) sk /= 2;
     }
     int st;
 #define MATQ_GEMV_T(RR, MT, NT, SK) launch_gemv_tensor<RR, MT, NT, SK>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
