@@ -9,8 +9,8 @@
 // The arithmetic of Eq. 1 is pinned to IEEE binary32 with one correctly
 // rounded operation per step (__fdiv_rn / __fadd_rn / __fsub_rn are never
 // contracted into FMAs), so the codes are reproducible bit for bit.  The
-// register-resident kernel reaches the same bits through a cheaper sequence
-// with a proven guard band and falls back to the pinned sequence inside it.
+// register-resident kernel reaches the same bits through a sequence of fused
+// multiply-adds that reproduces each of those roundings (see RowFast).
 #include "common.cuh"
 
 namespace matq {
@@ -81,46 +81,56 @@ __device__ __forceinline__ uint32_t codes_from_words(uint32_t w0, uint32_t w1, f
 
 // ---- the same codes without the special-function pipe ---------------------------------------------------------
 // Per element the pinned arithmetic needs a division, a floor and a float->int conversion, all of which issue on
-// the quarter-rate special-function pipe and bound the kernel.  The fast path below produces the SAME codes:
-//   u1 = fma(w, ra, z) with ra = correctly rounded 1/alpha (once per row): w * ra is within 2^-24 |t| of the exact
-//        quotient and the sum is rounded once, so u1 is within err = 2^-23 (2 |t| + |z|) of the pinned
-//        u = RN(RN(w / alpha) + z);
-//   r  = u1 rounded to the nearest integer with the 1.5 * 2^23 trick (no conversion instruction).
-// Rounding half up and rounding to nearest agree unless u sits on a tie, and u and u1 round alike unless u1 is within
-// err of a tie.  So whenever |u1 - r| < 1/2 - delta (delta = 4 err, a per-row constant) r IS the pinned result;
-// otherwise (about one element in a thousand) the element is recomputed with the pinned sequence.
+// the quarter-rate special-function pipe and bound the kernel.  The fast path below produces the SAME codes with
+// fused multiply-adds only, by reproducing every rounding of the pinned sequence:
+//   t = RN(w / alpha) from ra = RN(1 / alpha) (once per row) by two residual corrections
+//         q0 = RN(w ra),  r0 = w - q0 alpha (exact in an FMA),  q1 = RN(q0 + r0 ra)     (q1 is a faithful quotient)
+//         r1 = w - q1 alpha (exact),  t = RN(q1 + r1 ra)
+//       which is the correctly rounded quotient (Markstein's theorem: a faithful quotient corrected once with the
+//       exact residual and a correctly rounded reciprocal rounds correctly; rows whose alpha has an all-ones
+//       significand, the theorem's one exception, take the pinned path).  An FMA residual is only inexact when it
+//       underflows, i.e. for |w| below 2^-100: such a t is too small to move u = RN(t + z) across a rounding boundary.
+//   u = RN(t + z), exactly the pinned u.
+//   m = RN(u + 1.5 * 2^23) holds u rounded to the nearest-even integer in its low mantissa bits; u - (m - 1.5 * 2^23)
+//       is exact, and it equals +1/2 exactly when u was a tie that nearest-even rounded DOWN: round half up (the
+//       pinned rule) then gives one more.  Inside [0, 255] the code is the low byte of m's bit pattern, and u lies
+//       in [-2^-16, 255 + 2^-7] by construction of alpha and z, so no clamp and no conversion are needed.
+// Unlike a guard-band scheme this has no data-dependent fallback: with bf16 weights 0.2 % of the elements sit
+// exactly on a tie, enough to send a third of all warps down a divergent slow path.
 struct RowFast {
-    float a, z, ra, tie_guard;   // tie_guard = 1/2 - delta; <= 0 sends every element down the pinned path
+    float a, z, ra;
+    bool ok;        // false: the row is outside the fast path's domain and takes the pinned sequence
 };
 
-__device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx) {
-    RowFast f{a, z, 0.f, -1.f};
+__device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx, int bad) {
+    RowFast f{a, z, 0.f, false};
     const float big = fmaxf(fabsf(mn), fabsf(mx));
-    if (a > 1e-30f && a < 1e30f && fabsf(z) < 1048576.0f && big < 1e30f) {
+    if (!bad && a > 1e-30f && a < 1e30f && fabsf(z) < 1048576.0f && big < 1e30f &&
+        (__float_as_uint(a) & 0x007fffffu) != 0x007fffffu) {
         f.ra = __frcp_rn(a);
-        const float tmax = big * f.ra * 1.0001f;
-        const float delta = (2.0f * tmax + fabsf(z) + 1.0f) * 4.76837158e-7f;      // 4 * 2^-23 * (2 |t| + |z| + 1)
-        if (tmax + fabsf(z) < 2097152.0f) f.tie_guard = 0.5f - delta;              // |u| < 2^21: the rounding trick is exact
+        f.ok = big * f.ra * 1.0001f + fabsf(z) < 2097152.0f;      // |u| < 2^21: the rounding trick is exact
     }
     return f;
 }
 
-// Out of line on purpose: inlined, the compiler predicates the whole pinned sequence into the fast path and every
-// element pays for it; as a call it costs nothing unless a lane really is near a tie.
-__device__ __noinline__ float code_pinned(float w, float a, float z) { return code_from_weight(w, a, z); }
-
-__device__ __forceinline__ uint32_t code_fast(float w, const RowFast& f) {
-    const float u1 = __fmaf_rn(w, f.ra, f.z);                   // within err of the pinned u (see above)
-    const float m = __fadd_rn(u1, 12582912.0f);                 // 1.5 * 2^23: the sum is u1 rounded to an integer
-    const float r = __fsub_rn(m, 12582912.0f);
-    int code = __float_as_int(m) - 0x4b400000;                  // that integer, straight from the mantissa
-    if (!(fabsf(__fsub_rn(u1, r)) < f.tie_guard)) code = (int)code_pinned(w, f.a, f.z);   // near a tie (or NaN): pinned path
-    return (uint32_t)min(max(code, 0), 255);
-}
-
-__device__ __forceinline__ uint32_t codes_from_words_fast(uint32_t w0, uint32_t w1, const RowFast& f) {
-    return code_fast(__uint_as_float(w0 << 16), f) | (code_fast(__uint_as_float(w0 & 0xffff0000u), f) << 8) |
-           (code_fast(__uint_as_float(w1 << 16), f) << 16) | (code_fast(__uint_as_float(w1 & 0xffff0000u), f) << 24);
+// Eight codes of one 16-byte piece by the fast sequence.
+__device__ __forceinline__ uint2 codes8_fast(const uint4& v, const RowFast& f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t mb[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float x = __uint_as_float((j & 1) ? (w[j >> 1] & 0xffff0000u) : (w[j >> 1] << 16));
+        float q = __fmul_rn(x, f.ra);
+        q = __fmaf_rn(__fmaf_rn(-q, f.a, x), f.ra, q);
+        const float t = __fmaf_rn(__fmaf_rn(-q, f.a, x), f.ra, q);      // = RN(x / alpha)
+        const float u = __fadd_rn(t, f.z);
+        const float m = __fadd_rn(u, 12582912.0f);                      // 1.5 * 2^23
+        const float d = __fsub_rn(u, __fsub_rn(m, 12582912.0f));
+        mb[j] = __float_as_uint(m) + (d == 0.5f ? 1u : 0u);
+    }
+    const uint32_t lo = __byte_perm(__byte_perm(mb[0], mb[1], 0x0040), __byte_perm(mb[2], mb[3], 0x0040), 0x5410);
+    const uint32_t hi = __byte_perm(__byte_perm(mb[4], mb[5], 0x0040), __byte_perm(mb[6], mb[7], 0x0040), 0x5410);
+    return make_uint2(lo, hi);
 }
 
 // Fast path: K % 16 == 0, rows 16-byte aligned.  Dynamic shared memory: K * 2 bytes.
@@ -178,7 +188,7 @@ __device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& 
 // (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
 // folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
 template <int NV>
-__global__ void __launch_bounds__(kQuantThreads)
+__global__ void __launch_bounds__(kQuantThreads, NV <= 5 ? 4 : 2)
 quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw, int wpr,
                   uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
                   int32_t* dev_status) {
@@ -241,12 +251,19 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
         }
         if (q) {
             uint2* dst = reinterpret_cast<uint2*>(q + n * (int64_t)K);
-            const RowFast f = row_fast(a, z, mn, mx);
+            const RowFast f = row_fast(a, z, mn, mx, bad);
+            if (f.ok) {                                       // uniform over the row's team
 #pragma unroll
-            for (int j = 0; j < NV; ++j) {
-                const int i = team_tid + j * team_threads;
-                if (i < nvec)
-                    dst[i] = make_uint2(codes_from_words_fast(v[j].x, v[j].y, f), codes_from_words_fast(v[j].z, v[j].w, f));
+                for (int j = 0; j < NV; ++j) {
+                    const int i = team_tid + j * team_threads;
+                    if (i < nvec) dst[i] = codes8_fast(v[j], f);
+                }
+            } else {
+#pragma unroll 1
+                for (int i = team_tid; i < nvec; i += team_threads) {    // rare: re-read the row, pinned sequence
+                    const uint4 wv = ld_stream_u4(reinterpret_cast<const uint4*>(W + n * ldw) + i);
+                    dst[i] = make_uint2(codes_from_words(wv.x, wv.y, a, z), codes_from_words(wv.z, wv.w, a, z));
+                }
             }
         }
     }

@@ -78,6 +78,27 @@ def test_quantize_bit_exact_over_many_scales_and_offsets():
     assert np.abs(z_ref).max() > 2 ** 21                   # some rows did take the pinned path
 
 
+def test_quantize_bit_exact_on_every_bf16_numerator():
+    # The register kernel replaces the IEEE division by FMA corrections; this walks EVERY bf16 value between a row's
+    # extremes (8192 consecutive bit patterns per sign) for 256 different scales, alphas with all-ones and near-all-ones
+    # significands among them, so a quotient that is one ulp off anywhere would move a code.
+    rng = np.random.default_rng(7)
+    N, K = 256, 16384
+    W = np.empty((N, K), dtype=np.uint16)
+    for n in range(N):
+        top = int(rng.integers(0x2000, 0x5f00))                 # largest magnitude's bit pattern (about 1e-19 .. 1e19)
+        mags = np.arange(top - K // 2 + 1, top + 1, dtype=np.uint16)
+        W[n, : K // 2] = mags
+        W[n, K // 2:] = mags | 0x8000
+        if n % 4 == 1:
+            W[n, K // 2:] = mags[rng.integers(0, K // 2, K // 2)]   # same-sign row: another alpha, large z
+    st, q_ref, a_ref, z_ref = ref.quantize(W)
+    assert st == ref.OK
+    q, a, z = mq.quantize(bf16_dev(W))
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert np.array_equal(host(q), q_ref)
+
+
 def test_quantize_reports_nonfinite_without_trapping():
     Wf = synth.bf16_bits_to_f32(synth.normal_bf16((4, 128), 0.02, 9)).copy()
     Wf[2, 77] = np.inf
