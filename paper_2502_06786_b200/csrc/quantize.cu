@@ -187,15 +187,15 @@ __device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& 
 // Register-resident path (K <= 16384, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
 // (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
 // folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
-template <int NV>
-__global__ void __launch_bounds__(kQuantThreads, NV <= 5 ? 4 : 2)
+template <int NV, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, (NV <= 5 ? 32 : 16) / WARPS)
 quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw, int wpr,
                   uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
                   int32_t* dev_status) {
-    __shared__ float s_mn[kQuantThreads / 32], s_mx[kQuantThreads / 32];
-    __shared__ int s_bad[kQuantThreads / 32];
+    __shared__ float s_mn[WARPS], s_mx[WARPS];
+    __shared__ int s_bad[WARPS];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rows_per_cta = (kQuantThreads / 32) / wpr;
+    const int rows_per_cta = (WARPS) / wpr;
     const int team = warp / wpr, team_tid = (warp % wpr) * 32 + lane, team_threads = 32 * wpr;
     const int nvec = K >> 3;
     for (int64_t n_base = (int64_t)blockIdx.x * rows_per_cta; n_base < N; n_base += (int64_t)gridDim.x * rows_per_cta) {
@@ -321,10 +321,14 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
         int wpr = 1;
         while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 5) wpr *= 2;
         const int nv = (nvec + 32 * wpr - 1) / (32 * wpr);
-        const int rows_per_cta = 8 / wpr;
+        // CTAs of 4 warps when a row's team fits (measured 5 % faster than 8: more CTAs per SM in different phases)
+        const int warps = wpr <= 4 ? 4 : 8;
+        const int rows_per_cta = warps / wpr;
         int64_t grid = (N + rows_per_cta - 1) / rows_per_cta;
-        if (grid > (int64_t)sms * 16) grid = (int64_t)sms * 16;
-#define MATQ_QUANT_REG(NV) quantize_rows_reg<NV><<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status)
+        if (grid > (int64_t)sms * 32) grid = (int64_t)sms * 32;
+#define MATQ_QUANT_REG(NV) do { \
+        if (warps == 4) quantize_rows_reg<NV, 4><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status); \
+        else quantize_rows_reg<NV, 8><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status); } while (0)
         if (nv <= 2) MATQ_QUANT_REG(2);
         else if (nv <= 3) MATQ_QUANT_REG(3);
         else if (nv <= 4) MATQ_QUANT_REG(4);
