@@ -113,20 +113,56 @@ __device__ __forceinline__ RowFast row_fast(float a, float z, float mn, float mx
     return f;
 }
 
-// Eight codes of one 16-byte piece by the fast sequence.
+// Two fp32 lanes per instruction (sm_100 packed arithmetic; each lane rounds exactly like the scalar instruction).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// Eight codes of one 16-byte piece by the fast sequence, the two bf16 halves of a word side by side.
 __device__ __forceinline__ uint2 codes8_fast(const uint4& v, const RowFast& f) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const uint64_t ra2 = f2_pack(f.ra, f.ra), na2 = f2_pack(-f.a, -f.a), z2 = f2_pack(f.z, f.z);
+    const uint64_t c2 = f2_pack(12582912.0f, 12582912.0f);               // 1.5 * 2^23
     uint32_t mb[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float x = __uint_as_float((j & 1) ? (w[j >> 1] & 0xffff0000u) : (w[j >> 1] << 16));
-        float q = __fmul_rn(x, f.ra);
-        q = __fmaf_rn(__fmaf_rn(-q, f.a, x), f.ra, q);
-        const float t = __fmaf_rn(__fmaf_rn(-q, f.a, x), f.ra, q);      // = RN(x / alpha)
-        const float u = __fadd_rn(t, f.z);
-        const float m = __fadd_rn(u, 12582912.0f);                      // 1.5 * 2^23
-        const float d = __fsub_rn(u, __fsub_rn(m, 12582912.0f));
-        mb[j] = __float_as_uint(m) + (d == 0.5f ? 1u : 0u);
+    for (int j = 0; j < 4; ++j) {
+        const uint64_t x = f2_pack(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
+        uint64_t q = f2_mul(x, ra2);
+        q = f2_fma(f2_fma(q, na2, x), ra2, q);
+        const uint64_t t = f2_fma(f2_fma(q, na2, x), ra2, q);            // = RN(x / alpha)
+        const uint64_t u = f2_add(t, z2);
+        const uint64_t m = f2_add(u, c2);
+        const uint64_t d = f2_sub(u, f2_sub(m, c2));
+        float m0, m1, d0, d1;
+        f2_unpack(m, m0, m1);
+        f2_unpack(d, d0, d1);
+        mb[2 * j] = __float_as_uint(m0) + (d0 == 0.5f ? 1u : 0u);
+        mb[2 * j + 1] = __float_as_uint(m1) + (d1 == 0.5f ? 1u : 0u);
     }
     const uint32_t lo = __byte_perm(__byte_perm(mb[0], mb[1], 0x0040), __byte_perm(mb[2], mb[3], 0x0040), 0x5410);
     const uint32_t hi = __byte_perm(__byte_perm(mb[4], mb[5], 0x0040), __byte_perm(mb[6], mb[7], 0x0040), 0x5410);
