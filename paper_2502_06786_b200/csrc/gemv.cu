@@ -68,6 +68,12 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
 #define MATQ_GEMV_S(RR, MT, NT) ((sk == 8) ? MATQ_GEMV_T(RR, MT, NT, 8) : (sk == 4) ? MATQ_GEMV_T(RR, MT, NT, 4) : (sk == 2) ? MATQ_GEMV_T(RR, MT, NT, 2) : MATQ_GEMV_T(RR, MT, NT, 1))
 #define MATQ_GEMV_R(MT, NT) ((r == 8) ? MATQ_GEMV_S(8, MT, NT) : (r == 4) ? MATQ_GEMV_S(4, MT, NT) : MATQ_GEMV_S(2, MT, NT))
 #define MATQ_GEMV_RW(NT, W) ((r == 8) ? MATQ_GEMV_W(8, NT, W) : (r == 4) ? MATQ_GEMV_W(4, NT, W) : MATQ_GEMV_W(2, NT, W))
+    const bool wide = mt == 2 && sk == 8 && B > 4 && B <= 8 && ((N + 31) / 32 + 1) / 2 <= sms;
+    if (wide) {                    // a batch: 16-warp CTAs (two row tiles) halve the staging of x' per SM (measured 4-12 %)
+        st = (r == 8) ? launch_gemv_tensor<8, 2, 1, 8, 16>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+           : (r == 4) ? launch_gemv_tensor<4, 2, 1, 8, 16>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+                      : launch_gemv_tensor<2, 2, 1, 8, 16>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+    } else
     if (sk >= 16) {                // few, long rows: one 16-row tile per CTA, K split over 16 or 32 warps
         if (B <= 8) st = (sk == 32) ? MATQ_GEMV_RW(1, 32) : MATQ_GEMV_RW(1, 16);
         else st = (sk == 32) ? MATQ_GEMV_RW(2, 32) : MATQ_GEMV_RW(2, 16);
