@@ -265,17 +265,21 @@ gemv_tensor(const GemvTensorParams P) {
         // Item i = ((q*4 + j) * bpad + gg) * 4 + tt covers one packed word's worth of activations.  (i >> 2) % bpad
         // is the batch column and threads / 4 is a multiple of bpad, so every group of 4 lanes sees a single column.
         {
-            const int items = (pass_hi - pass_lo) * 4 * bpad * 4;
-            const int qj0 = pass_lo * 4;
-            for (int i = tid; i < items; i += kGemvThreads) {
-                const int tt = i & 3;
-                const int gg = (i >> 2) & (bpad - 1);        // bpad is a power of two
-                const int qjl = (i >> 2) >> P.bpad_log2;     // (q - pass_lo)*4 + j
-                const int qj = qj0 + qjl;
-                const int64_t kb = (int64_t)(qj >> 2) * kWq + tt * (kWq / 4) + (qj & 3) * Fmt::kWeightsPerWord;
-                uint4* dst = xs + ((size_t)qjl * kPG * bpad + gg) * 4 + tt;
-                if (gg < P.B && kb < P.K) {                   // K % 128 == 0: a word lies inside or outside
-                    stage_word<R>(P.x + (int64_t)gg * P.ldx + kb, dst, bpad * 4, sx, sxp);
+            // thread -> (tt, gg) is fixed; its items are qstep apart in (q*4 + j), so everything but two adds is hoisted
+            const int n_qjl = (pass_hi - pass_lo) * 4;
+            const int qstep = (kGemvThreads / 4) >> P.bpad_log2;
+            const int tt = tid & 3, gg = (tid >> 2) & (bpad - 1);
+            const bool col_ok = gg < P.B;
+            const __nv_bfloat16* xrow = P.x + (int64_t)(col_ok ? gg : 0) * P.ldx;
+            int qjl = (tid >> 2) >> P.bpad_log2;
+            uint4* dst = xs + ((uint32_t)qjl * kPG * bpad + gg) * 4 + tt;
+            const uint32_t dstep = (uint32_t)qstep * kPG * bpad * 4;
+            const int kmax = (int)P.K;
+            for (; qjl < n_qjl; qjl += qstep, dst += dstep) {
+                const int qj = pass_lo * 4 + qjl;
+                const int kb = Fmt::kWeightsPerWord * (16 * (qj >> 2) + 4 * tt + (qj & 3));
+                if (col_ok && kb < kmax) {                    // K % 128 == 0: a word lies inside or outside
+                    stage_word<R>(xrow + kb, dst, bpad * 4, sx, sxp);
                 } else {
                     dst[0] = make_uint4(0, 0, 0, 0);
                     if (kPG == 2) dst[bpad * 4] = make_uint4(0, 0, 0, 0);
