@@ -187,20 +187,23 @@ gemv_tensor(const GemvTensorParams P) {
     float* part = reinterpret_cast<float*>(smem_raw + (size_t)min(P.qc_pass, P.n_qc) * 4 * kPG * bpad * 64);
 
     // ---- weights of the first chunks are requested before anything that depends on the previous kernel
+    // Rows past N are clamped to the last row (their results are never stored) and a lane whose piece would start
+    // past the end of a ragged last chunk is clamped to the row's last 16 bytes (the matching activations are staged
+    // as zeros and unpacked fields are always finite), so the loads need no predicates and no zero fill.
     const uint8_t* wrow[2 * MT];
     bool wok[2 * MT];
 #pragma unroll
     for (int h = 0; h < 2 * MT; ++h) {
         const int64_t row = row0 + (h >> 1) * 16 + (h & 1) * 8 + g;
         wok[h] = row < P.N;
-        wrow[h] = P.packed + (wok[h] ? row : 0) * P.row_bytes + t * 16;
+        wrow[h] = P.packed + (wok[h] ? row : P.N - 1) * P.row_bytes;
     }
+    const int max_off = (int)P.row_bytes - 16;
     auto load_chunk = [&](int q, uint4 (&dst)[2 * MT]) {
-        const bool in = q < q_hi && (int64_t)q * 64 + t * 16 < P.row_bytes;
+        if (q < q_hi) {                                   // warp-uniform
+            const int off = min(q * 64 + t * 16, max_off);
 #pragma unroll
-        for (int h = 0; h < 2 * MT; ++h) {
-            dst[h] = make_uint4(0, 0, 0, 0);
-            if (in && wok[h]) dst[h] = ld_stream_u4(wrow[h] + (int64_t)q * 64);
+            for (int h = 0; h < 2 * MT; ++h) dst[h] = ld_stream_u4(wrow[h] + off);
         }
     };
     uint4 wbuf[kGemvDepth][2 * MT];
@@ -444,6 +447,7 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     P.x = static_cast<const __nv_bfloat16*>(x); P.y = y;
     P.N = N; P.K = K; P.ldx = ldx; P.ldy = ldy;
     P.row_bytes = K * R / 8;
+    if (P.row_bytes > 0x7fffffff) return MATQ_ERR_SHAPE;   // byte offsets inside a row are 32-bit
     P.B = B;
     P.bpad = B <= 1 ? 1 : B <= 2 ? 2 : B <= 4 ? 4 : B <= 8 ? 8 : 16;
     P.n_qc = (int)((P.row_bytes + 63) / 64);
