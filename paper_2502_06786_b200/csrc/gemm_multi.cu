@@ -57,6 +57,8 @@ __device__ __forceinline__ uint64_t sw128_desc(uint32_t smem_addr) {
 }
 // kind::f16, D = fp32, A = B = bf16, both K-major, N = 128, M = 128
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// the same with N = 256: two adjacent plane tiles in one instruction
+constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * kBN) >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_b0,
@@ -135,11 +137,15 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
                 for (int kk = 0; kk < kBK / 16; ++kk) {
                     const uint64_t ad = sw128_desc(a_base + kk * 32);
+                    // The tiles of the first two planes are adjacent in the stage (rows 0..255 of one K-major operand) and
+                    // so are their accumulators in TMEM: one N = 256 MMA covers both and reads the X tile once for them.
+                    const uint32_t accumulate = (kb > 0 || kk > 0) ? 1u : 0u;
                     for (int r = 0; r < P.n_r; ++r) {
+                        const bool pair = (r == 0 && P.n_r >= 2);
                         const uint64_t bd = sw128_desc(a_base + (1 + r) * kTileBytes + kk * 32);
-                        const uint32_t accumulate = (kb > 0 || kk > 0) ? 1u : 0u;
                         asm volatile("{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
-                                     ::"r"(tmem + r * kBN), "l"(ad), "l"(bd), "r"(kIdesc), "r"(accumulate) : "memory");
+                                     ::"r"(tmem + r * kBN), "l"(ad), "l"(bd), "r"(pair ? kIdesc2 : kIdesc), "r"(accumulate) : "memory");
+                        if (pair) ++r;
                     }
                 }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_empty[s])) : "memory");
