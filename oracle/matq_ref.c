@@ -129,6 +129,62 @@ int matq_ref_quantize(const uint16_t *W, int64_t N, int64_t K, int64_t ldw, int 
     return bad ? MATQ_REF_ERR_NONFINITE : MATQ_REF_OK;
 }
 
+/* ------------------------------------------------------------------ Eq. 3 */
+/* MinMax quantisation with OmniQuant's two clipping scales (Section 3.1, Eq. 3):
+ *   alpha = (gamma * max(w) - beta * min(w)) / (2^c - 1),  z = -beta * min(w) / alpha,
+ *   Q = clamp(round(w / alpha + z), 0, 2^c - 1),
+ * gamma and beta per output channel (NULL = 1 for every row, which is Eq. 1).
+ * Every step is one fp32 operation, in the order written: the two products,
+ * their difference, the division by 2^c - 1, the division for z, then per weight
+ * the division, the sum, round half up and the clamp.  A range that is not
+ * positive gives alpha = 1 (the reading taken for a constant row in Eq. 1).
+ * A non-finite weight, gamma or beta makes the call return
+ * MATQ_REF_ERR_NONFINITE (that row's outputs are then unspecified). */
+int matq_ref_quantize_clip(const uint16_t *W, int64_t N, int64_t K, int64_t ldw, int c,
+                           const float *gamma, const float *beta,
+                           uint8_t *q, float *alpha, float *zero)
+{
+    if (!W || !alpha || !zero || N < 0 || K <= 0 || ldw < K) return MATQ_REF_ERR_INVALID_ARG;
+    if (c != 8) return MATQ_REF_ERR_UNSUPPORTED;
+    const float qmax = (float)((1 << c) - 1);
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (int64_t n = 0; n < N; ++n) {
+        const uint16_t *row = W + n * ldw;
+        float mn = bf16_to_float(row[0]);
+        float mx = mn;
+        int nonfinite = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float w = bf16_to_float(row[k]);
+            if (!isfinite(w)) nonfinite = 1;
+            if (w < mn) mn = w;
+            if (w > mx) mx = w;
+        }
+        const float g = gamma ? gamma[n] : 1.0f;
+        const float b = beta ? beta[n] : 1.0f;
+        if (!isfinite(g) || !isfinite(b)) nonfinite = 1;
+        if (nonfinite) { bad |= 1; continue; }
+        float hi = g * mx;
+        float lo = b * mn;
+        float range = hi - lo;
+        float a = (range > 0.0f) ? range / qmax : 1.0f;
+        float z = (-lo) / a;
+        alpha[n] = a;
+        zero[n] = z;
+        if (!q) continue;
+        for (int64_t k = 0; k < K; ++k) {
+            float w = bf16_to_float(row[k]);
+            float t = w / a;
+            float u = t + z;
+            float r = round_half_up(u);
+            if (r < 0.0f) r = 0.0f;
+            if (r > qmax) r = qmax;
+            q[n * K + k] = (uint8_t)r;
+        }
+    }
+    return bad ? MATQ_REF_ERR_NONFINITE : MATQ_REF_OK;
+}
+
 /* ------------------------------------------------------- Eq. 6 and Eq. 8 */
 /* Value of S(q, r) on the c-bit grid, 0 .. 2^c (2^c only with Eq. 8).
  * floor(q / 2^sh + 1/2) on integers is (q + 2^(sh-1)) >> sh. */

@@ -66,6 +66,22 @@ def quantize(W_bits: np.ndarray, c: int = 8, want_codes: bool = True):
     return st, q, alpha, zero
 
 
+def quantize_clip(W_bits: np.ndarray, gamma=None, beta=None, c: int = 8, want_codes: bool = True):
+    """Eq. 3 per row (gamma, beta fp32 [N] or None = 1).  Returns (status, q or None, alpha, zero)."""
+    _chk(W_bits, np.uint16, "W")
+    N, K = W_bits.shape
+    if gamma is not None:
+        _chk(gamma, np.float32, "gamma")
+    if beta is not None:
+        _chk(beta, np.float32, "beta")
+    q = np.empty((N, K), np.uint8) if want_codes else None
+    alpha = np.zeros(N, np.float32)
+    zero = np.zeros(N, np.float32)
+    st = lib().matq_ref_quantize_clip(_p(W_bits), C.c_int64(N), C.c_int64(K), C.c_int64(K), C.c_int(c),
+                                      _p(gamma), _p(beta), _p(q), _p(alpha), _p(zero))
+    return st, q, alpha, zero
+
+
 def slice_values(q: np.ndarray, r: int, extra_precision: bool = False, c: int = 8):
     """Eq. 6 (or Eq. 8) elementwise.  Returns (status, S uint16, same shape)."""
     _chk(q, np.uint8, "q")
