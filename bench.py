@@ -362,6 +362,8 @@ def run_cuda(args, rank, world, local_rank):
         cfg4 = gemm_cfg4(mq, torch, peaks)
         torch.cuda.empty_cache()
         extras = {"gemv_cfg3": gemv_cfg3(mq, torch, peaks), "gemm_multi_cfg5_prefill": gemm_cfg5_prefill(mq, torch, peaks)}
+        torch.cuda.empty_cache()
+        extras["quantize_clip_cfg5"] = quantize_clip_cfg5(mq, torch, peaks)
 
     out = None
     if rank == 0:
@@ -453,6 +455,44 @@ def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
         del planes, xs, ys, al, g
         torch.cuda.empty_cache()
     return out
+
+
+def quantize_clip_cfg5(mq, torch, peaks, layers=2, reps=10):
+    """Eq. 3 on configs[4]'s weights: Gemma-2-9B MLP shapes, Student-t(3) weights, clipping scales gamma = beta = 0.5
+    on every channel (learning them is outside the library), then the extra-precision int2 slice of those codes:
+    the fraction of codes in the extra bucket comes from the weights and the clamp, not from injected codes."""
+    shapes = [(n, k) for _ in range(layers) for (_, n, k) in synth.gemma2_9b_mlp_layer()]
+    Ws = [torch.from_numpy(synth.weight_bf16(5, i, n, k)).cuda().view(torch.bfloat16) for i, (n, k) in enumerate(shapes)]
+    outs = [(torch.empty((n, k), dtype=torch.uint8, device="cuda"), torch.empty(n, device="cuda"), torch.empty(n, device="cuda"))
+            for n, k in shapes]
+    gs = [torch.full((n,), 0.5, device="cuda") for n, k in shapes]
+
+    def run():
+        for W, (q, a, z), g in zip(Ws, outs, gs):
+            mq.quantize(W, q=q, alpha=a, zero=z, gamma=g, beta=g)
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            run()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    nbytes = sum(bytes_quantize(n, k) + 8 * n for n, k in shapes)
+    n0, k0 = shapes[0]
+    sp = mq.slice_pack(outs[0][0], 2, extra_precision=True, ovf_capacity=n0 * k0)
+    return {"workload": f"Eq. 3 on configs[4] weights: {layers} Gemma-2-9B MLP layers, Student-t(3), gamma = beta = 0.5, matq_quantize_clip",
+            "ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1), "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4),
+            "launches": len(shapes), "overflow_fraction_r2": round(int(sp["ovf_count"].item()) / (n0 * k0), 4)}
 
 
 def gemm_cfg5_prefill(mq, torch, peaks, reps=3):

@@ -94,6 +94,24 @@ int matq_quantize(const void *W, int64_t N, int64_t K, int64_t ldw, int c,
                   int32_t *dev_status, void *stream);
 
 /*
+ * (1b) MinMax quantisation with OmniQuant's two clipping scales per output channel (Section 3.1, Eq. 3):
+ *       alpha_n = (gamma_n max_k W[n,k] - beta_n min_k W[n,k]) / (2^c - 1),  z_n = -beta_n min_k W[n,k] / alpha_n,
+ *       q[n,k]  = clamp(round_half_up(W[n,k] / alpha_n + z_n), 0, 2^c - 1)
+ *     in IEEE binary32, one correctly rounded operation per step in the order written (the two products, their
+ *     difference, the division by 2^c - 1, the division for z, then per weight as in Eq. 1).  Scales below 1 clip
+ *     the range: weights outside it saturate at 0 or 2^c - 1, which is what fills the top bucket that the
+ *     extra-precision slice (Eq. 8) keeps.  gamma_n max - beta_n min <= 0 gives alpha = 1, z = -beta_n min.
+ *   gamma, beta  in  fp32 [N] device pointers; either may be NULL (= 1 for every row; both NULL is matq_quantize)
+ *   A non-finite weight or scale sets dev_status = MATQ_ERR_NONFINITE; that row's outputs are unspecified.
+ *   Everything else (W, q, alpha, zero, shapes, alignment, errors) as for matq_quantize.  How gamma and beta are
+ *   learned is outside this library.
+ */
+int matq_quantize_clip(const void *W, int64_t N, int64_t K, int64_t ldw, int c,
+                       const float *gamma, const float *beta,
+                       uint8_t *q, float *alpha, float *zero,
+                       int32_t *dev_status, void *stream);
+
+/*
  * (2) MSB slicing S(q, r) of Eq. 6 (extra_precision = 0) or of the Errata's
  *     Eq. 8 (extra_precision = 1), then packing.  With sh = c - r:
  *       k      = min((q + 2^(sh-1)) >> sh, 2^r - 1)      (k = q when sh = 0)

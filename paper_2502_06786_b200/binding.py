@@ -21,7 +21,7 @@ ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_CAPACITY, ERR_TIMEOUT = 5, 6, 8, 9, 
 SRC_BF16, SRC_CODES8, SRC_PACKED = 0, 1, 2
 GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_PDL = 0, 1, 2, 3, 0x100
 
-EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize",
+EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
            "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
@@ -47,6 +47,8 @@ def _load():
     lib.matq_packed_row_bytes.argtypes = [i64, i32]
     lib.matq_quantize.restype = i32
     lib.matq_quantize.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, vp]
+    lib.matq_quantize_clip.restype = i32
+    lib.matq_quantize_clip.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.matq_slice_pack.restype = i32
     lib.matq_slice_pack.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, i64, vp, vp, vp]
     lib.matq_gemv_workspace_bytes.restype = sz
@@ -112,8 +114,9 @@ def _check(st, where, raise_on_error=True):
     return st
 
 
-def quantize(W, q=None, alpha=None, zero=None, dev_status=None, want_codes=True, c=8):
-    """matq_quantize.  W: bf16 [N, K] (row stride W.stride(0)).  Returns (q, alpha, zero)."""
+def quantize(W, q=None, alpha=None, zero=None, dev_status=None, want_codes=True, c=8, gamma=None, beta=None):
+    """matq_quantize, or matq_quantize_clip when gamma / beta (fp32 [N], Eq. 3's clipping scales) are given.
+    W: bf16 [N, K] (row stride W.stride(0)).  Returns (q, alpha, zero)."""
     _dev(W, torch.bfloat16, "W", 2)
     if W.stride(1) != 1:
         raise ValueError("W: unit stride along K required")
@@ -125,9 +128,19 @@ def quantize(W, q=None, alpha=None, zero=None, dev_status=None, want_codes=True,
         alpha = torch.empty(N, dtype=torch.float32, device=dev)
     if zero is None:
         zero = torch.empty(N, dtype=torch.float32, device=dev)
-    st = _lib.matq_quantize(_ptr(W), N, K, _ld(W, K), c, _ptr(q), _ptr(alpha), _ptr(zero),
-                            _ptr(dev_status), _stream())
-    _check(st, "matq_quantize")
+    if gamma is None and beta is None:
+        st = _lib.matq_quantize(_ptr(W), N, K, _ld(W, K), c, _ptr(q), _ptr(alpha), _ptr(zero),
+                                _ptr(dev_status), _stream())
+        _check(st, "matq_quantize")
+    else:
+        for name, t in (("gamma", gamma), ("beta", beta)):
+            if t is not None:
+                _dev(t, torch.float32, name, 1)
+                if t.numel() != N or not t.is_contiguous():
+                    raise ValueError(f"{name}: contiguous fp32 [N] required")
+        st = _lib.matq_quantize_clip(_ptr(W), N, K, _ld(W, K), c, _ptr(gamma), _ptr(beta), _ptr(q), _ptr(alpha),
+                                     _ptr(zero), _ptr(dev_status), _stream())
+        _check(st, "matq_quantize_clip")
     return q, alpha, zero
 
 

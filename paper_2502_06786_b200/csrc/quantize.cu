@@ -57,10 +57,21 @@ __device__ __forceinline__ RowRange block_range(float mn, float mx, int bad) {
     return r;
 }
 
-__device__ __forceinline__ void scale_zero(const RowRange& rr, float& a, float& z) {
-    const float range = __fsub_rn(rr.mx, rr.mn);
+// alpha and z of Eq. 3 from the row's extremes and its clipping scales (g = b = 1 is Eq. 1 exactly: the products
+// are then exact).  One correctly rounded operation per step, in the order the header states.
+__device__ __forceinline__ void scale_zero(const RowRange& rr, float g, float b, float& a, float& z) {
+    const float hi = __fmul_rn(g, rr.mx), lo = __fmul_rn(b, rr.mn);
+    const float range = __fsub_rn(hi, lo);
     a = (range > 0.0f) ? __fdiv_rn(range, 255.0f) : 1.0f;
-    z = __fdiv_rn(-rr.mn, a);
+    z = __fdiv_rn(-lo, a);
+}
+
+// Clipping scales of row n (absent = 1); a non-finite scale marks the row bad like a non-finite weight.
+__device__ __forceinline__ void row_scales(const float* __restrict__ gamma, const float* __restrict__ beta, int64_t n,
+                                           float& g, float& b, int& bad) {
+    g = gamma ? gamma[n] : 1.0f;
+    b = beta ? beta[n] : 1.0f;
+    bad |= !(fabsf(g) <= 3.4e38f) | !(fabsf(b) <= 3.4e38f);
 }
 
 __device__ __forceinline__ void fold_word(uint32_t w, float& mn, float& mx, int& bad) {
@@ -143,7 +154,9 @@ __device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
     return r;
 }
 
-// Eight codes of one 16-byte piece by the fast sequence, the two bf16 halves of a word side by side.
+// Eight codes of one 16-byte piece by the fast sequence, the two bf16 halves of a word side by side.  CLIP: Eq. 3's
+// scales can put u outside [0, 255]; rounding is monotone, so clamping u first gives the clamped code.
+template <bool CLIP>
 __device__ __forceinline__ uint2 codes8_fast(const uint4& v, const RowFast& f) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     const uint64_t ra2 = f2_pack(f.ra, f.ra), na2 = f2_pack(-f.a, -f.a), z2 = f2_pack(f.z, f.z);
@@ -155,7 +168,12 @@ __device__ __forceinline__ uint2 codes8_fast(const uint4& v, const RowFast& f) {
         uint64_t q = f2_mul(x, ra2);
         q = f2_fma(f2_fma(q, na2, x), ra2, q);
         const uint64_t t = f2_fma(f2_fma(q, na2, x), ra2, q);            // = RN(x / alpha)
-        const uint64_t u = f2_add(t, z2);
+        uint64_t u = f2_add(t, z2);
+        if (CLIP) {
+            float u0, u1;
+            f2_unpack(u, u0, u1);
+            u = f2_pack(fminf(fmaxf(u0, 0.0f), 255.0f), fminf(fmaxf(u1, 0.0f), 255.0f));
+        }
         const uint64_t m = f2_add(u, c2);
         const uint64_t d = f2_sub(u, f2_sub(m, c2));
         float m0, m1, d0, d1;
@@ -172,6 +190,7 @@ __device__ __forceinline__ uint2 codes8_fast(const uint4& v, const RowFast& f) {
 // Fast path: K % 16 == 0, rows 16-byte aligned.  Dynamic shared memory: K * 2 bytes.
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
+                  const float* __restrict__ gamma, const float* __restrict__ beta,
                   uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
                   int32_t* dev_status) {
     extern __shared__ uint4 row_s[];
@@ -188,9 +207,10 @@ quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
             fold_word(v.z, mn, mx, bad);
             fold_word(v.w, mn, mx, bad);
         }
-        const RowRange rr = block_range(mn, mx, bad);   // its barriers also publish row_s
-        float a, z;
-        scale_zero(rr, a, z);
+        RowRange rr = block_range(mn, mx, bad);         // its barriers also publish row_s
+        float a, z, g, b;
+        row_scales(gamma, beta, n, g, b, rr.bad);
+        scale_zero(rr, g, b, a, z);
         if (threadIdx.x == 0) {
             if (rr.bad) report(dev_status, MATQ_ERR_NONFINITE);
             alpha[n] = a;
@@ -223,9 +243,10 @@ __device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& 
 // Register-resident path (K <= 16384, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
 // (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
 // folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
-template <int NV, int WARPS>
+template <int NV, int WARPS, bool CLIP>
 __global__ void __launch_bounds__(WARPS * 32, (NV <= 5 ? 32 : 16) / WARPS)
 quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw, int wpr,
+                  const float* __restrict__ gamma, const float* __restrict__ beta,
                   uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
                   int32_t* dev_status) {
     __shared__ float s_mn[WARPS], s_mx[WARPS];
@@ -277,9 +298,10 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
             }
         }
         if (!live) continue;
+        float a, z, g, b;
+        row_scales(gamma, beta, n, g, b, bad);
         RowRange rr{mn, mx, bad};
-        float a, z;
-        scale_zero(rr, a, z);
+        scale_zero(rr, g, b, a, z);
         if (team_tid == 0) {
             if (bad) report(dev_status, MATQ_ERR_NONFINITE);
             alpha[n] = a;
@@ -292,7 +314,7 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
 #pragma unroll
                 for (int j = 0; j < NV; ++j) {
                     const int i = team_tid + j * team_threads;
-                    if (i < nvec) dst[i] = codes8_fast(v[j], f);
+                    if (i < nvec) dst[i] = codes8_fast<CLIP>(v[j], f);
                 }
             } else {
 #pragma unroll 1
@@ -308,6 +330,7 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
 // Any K, ldw, alignment: scalar loads, the row is read twice (second pass usually from L2).
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_rows_generic(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
+                      const float* __restrict__ gamma, const float* __restrict__ beta,
                       uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
                       int32_t* dev_status) {
     for (int64_t n = blockIdx.x; n < N; n += gridDim.x) {
@@ -321,9 +344,10 @@ quantize_rows_generic(const uint16_t* __restrict__ W, int64_t N, int64_t K, int6
             mx = fmaxf(mx, w);
             bad |= ((b & 0x7f80u) == 0x7f80u);
         }
-        const RowRange rr = block_range(mn, mx, bad);
-        float a, z;
-        scale_zero(rr, a, z);
+        RowRange rr = block_range(mn, mx, bad);
+        float a, z, g, b;
+        row_scales(gamma, beta, n, g, b, rr.bad);
+        scale_zero(rr, g, b, a, z);
         if (threadIdx.x == 0) {
             if (rr.bad) report(dev_status, MATQ_ERR_NONFINITE);
             alpha[n] = a;
@@ -341,7 +365,15 @@ quantize_rows_generic(const uint16_t* __restrict__ W, int64_t N, int64_t K, int6
 extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, int c,
                              uint8_t* q, float* alpha, float* zero,
                              int32_t* dev_status, void* stream) {
+    return matq_quantize_clip(W, N, K, ldw, c, nullptr, nullptr, q, alpha, zero, dev_status, stream);
+}
+
+extern "C" int matq_quantize_clip(const void* W, int64_t N, int64_t K, int64_t ldw, int c,
+                                  const float* gamma, const float* beta,
+                                  uint8_t* q, float* alpha, float* zero,
+                                  int32_t* dev_status, void* stream) {
     using namespace matq;
+    const bool clip = gamma != nullptr || beta != nullptr;
     if (N < 0 || K <= 0 || ldw < K || (N > 0 && (!W || !alpha || !zero))) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     if (N == 0) return MATQ_OK;
@@ -363,8 +395,13 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
         int64_t grid = (N + rows_per_cta - 1) / rows_per_cta;
         if (grid > (int64_t)sms * 32) grid = (int64_t)sms * 32;
 #define MATQ_QUANT_REG(NV) do { \
-        if (warps == 4) quantize_rows_reg<NV, 4><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status); \
-        else quantize_rows_reg<NV, 8><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, q, alpha, zero, dev_status); } while (0)
+        if (clip) { \
+            if (warps == 4) quantize_rows_reg<NV, 4, true><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            else quantize_rows_reg<NV, 8, true><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+        } else { \
+            if (warps == 4) quantize_rows_reg<NV, 4, false><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            else quantize_rows_reg<NV, 8, false><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+        } } while (0)
         if (nv <= 2) MATQ_QUANT_REG(2);
         else if (nv <= 3) MATQ_QUANT_REG(3);
         else if (nv <= 4) MATQ_QUANT_REG(4);
@@ -379,10 +416,10 @@ extern "C" int matq_quantize(const void* W, int64_t N, int64_t K, int64_t ldw, i
         int per_sm = (int)((200u * 1024u) / (smem + 1024));
         per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
         const int64_t grid = N < (int64_t)sms * per_sm ? N : (int64_t)sms * per_sm;
-        quantize_rows_vec<<<(unsigned)grid, kQuantThreads, smem, s>>>(Wb, N, (int)K, ldw, q, alpha, zero, dev_status);
+        quantize_rows_vec<<<(unsigned)grid, kQuantThreads, smem, s>>>(Wb, N, (int)K, ldw, gamma, beta, q, alpha, zero, dev_status);
     } else {
         const int64_t grid = N < (int64_t)sms * 8 ? N : (int64_t)sms * 8;
-        quantize_rows_generic<<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, K, ldw, q, alpha, zero, dev_status);
+        quantize_rows_generic<<<(unsigned)grid, kQuantThreads, 0, s>>>(Wb, N, K, ldw, gamma, beta, q, alpha, zero, dev_status);
     }
     return launch_status();
 }

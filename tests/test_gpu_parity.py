@@ -99,6 +99,53 @@ def test_quantize_bit_exact_on_every_bf16_numerator():
     assert np.array_equal(host(q), q_ref)
 
 
+@pytest.mark.parametrize("N,K,dist", [(9216, 2304, "normal"), (300, 9216, "student"), (64, 4096, "student"), (33, 16384, "normal"),
+                                      (19, 1000, "normal"), (7, 72, "student"), (2304, 9216, "normal"), (6, 77, "normal"), (9, 32768, "student")])
+def test_quantize_clip_bit_exact(N, K, dist):
+    # Eq. 3: per-channel clipping scales; every kernel variant (register, shared-memory and scalar paths) against the oracle
+    W = synth.normal_bf16((N, K), 0.02, 900 + N) if dist == "normal" else synth.student_t_bf16((N, K), 3.0, 0.02, 950 + N)
+    rng = np.random.default_rng(N + K)
+    gamma = rng.uniform(0.4, 1.0, N).astype(np.float32)
+    beta = rng.uniform(0.4, 1.0, N).astype(np.float32)
+    gamma[::5] = 1.0
+    beta[1::7] = 1.0
+    if N > 4:
+        gamma[2], beta[2] = 0.0, 0.0                     # degenerate range: alpha = 1
+        gamma[3], beta[3] = 1.5, 1.25                    # scales above 1 widen the range
+    st, q_ref, a_ref, z_ref = ref.quantize_clip(W, gamma, beta)
+    assert st == ref.OK
+    status = status_word()
+    q, a, z = mq.quantize(bf16_dev(W), gamma=dev(gamma), beta=dev(beta), dev_status=status)
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert np.array_equal(host(q), q_ref)
+    assert int(host(status)[0]) == mq.OK
+    assert (q_ref == 255).any() and (q_ref == 0).any()
+    # only one of the two scales
+    st, q_ref, a_ref, z_ref = ref.quantize_clip(W, None, beta)
+    q, a, z = mq.quantize(bf16_dev(W), beta=dev(beta))
+    assert np.array_equal(host(q), q_ref) and np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+
+
+def test_quantize_clip_on_every_bf16_numerator_and_nonfinite_scale():
+    rng = np.random.default_rng(11)
+    N, K = 64, 16384
+    W = np.empty((N, K), dtype=np.uint16)
+    for n in range(N):
+        top = int(rng.integers(0x3000, 0x4f00))
+        mags = np.arange(top - K // 2 + 1, top + 1, dtype=np.uint16)
+        W[n, : K // 2] = mags
+        W[n, K // 2:] = mags | 0x8000
+    gamma = rng.uniform(0.05, 1.0, N).astype(np.float32)
+    beta = rng.uniform(0.05, 1.0, N).astype(np.float32)
+    st, q_ref, a_ref, z_ref = ref.quantize_clip(W, gamma, beta)
+    q, a, z = mq.quantize(bf16_dev(W), gamma=dev(gamma), beta=dev(beta))
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref) and np.array_equal(host(q), q_ref)
+    gamma[5] = np.nan
+    status = status_word()
+    mq.quantize(bf16_dev(W), gamma=dev(gamma), beta=dev(beta), dev_status=status)
+    assert int(host(status)[0]) == mq.ERR_NONFINITE
+
+
 def test_quantize_reports_nonfinite_without_trapping():
     Wf = synth.bf16_bits_to_f32(synth.normal_bf16((4, 128), 0.02, 9)).copy()
     Wf[2, 77] = np.inf
