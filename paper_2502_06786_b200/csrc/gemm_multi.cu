@@ -38,6 +38,7 @@ struct Params {
     int sh[kMaxR];
     int64_t M, N, K, ldy;
     int n_r, stages;
+    int wide;      // one plane only: the CTA takes 256 channels as two adjacent 128-row tiles (n_r is then 2)
     int32_t* dev_status;
 };
 
@@ -66,14 +67,14 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_acc;
     __shared__ uint32_t s_tmem;
-    __shared__ float s_alpha[kBN], s_az[kBN];              // alpha_n and alpha_n * z_n of this tile's columns
+    __shared__ float s_alpha[2 * kBN], s_az[2 * kBN];      // alpha_n and alpha_n * z_n of this tile's columns
     __shared__ int s_timeout;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // blockIdx.x walks the token tiles: CTAs that run together share one 128-channel slab of the planes (3 x 1 MB,
     // read from HBM once) and differ in their X tiles, and all of X stays in the L2.  The other order re-streams the
     // planes from HBM once per token tile.
-    const int64_t m0 = (int64_t)blockIdx.x * kBM, n0 = (int64_t)blockIdx.y * kBN;
+    const int64_t m0 = (int64_t)blockIdx.x * kBM, n0 = (int64_t)blockIdx.y * (P.wide ? 2 * kBN : kBN);
     const int nkb = (int)(P.K / kBK);
     const int stage_bytes = (1 + P.n_r) * kTileBytes;
     const int tmem_cols = P.n_r == 1 ? 128 : (P.n_r == 2 ? 256 : 512);
@@ -94,11 +95,12 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (warp >= 2) {
-        const int c = tid - 64;                              // 0..127: a column of this tile
-        const int64_t n = n0 + c;
-        const float a = n < P.N ? P.alpha[n] : 0.f, z = n < P.N ? P.zero[n] : 0.f;
-        s_alpha[c] = a;
-        s_az[c] = a * z;
+        for (int c = tid - 64; c < (P.wide ? 2 * kBN : kBN); c += kBN) {   // a column of this tile
+            const int64_t n = n0 + c;
+            const float a = n < P.N ? P.alpha[n] : 0.f, z = n < P.N ? P.zero[n] : 0.f;
+            s_alpha[c] = a;
+            s_az[c] = a * z;
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -121,7 +123,8 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                              ::"r"(smem_u32(st)), "l"(&tm_x), "r"(k0), "r"((int)m0), "r"(bar) : "memory");
                 for (int r = 0; r < P.n_r; ++r)
                     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                                 ::"r"(smem_u32(st + (size_t)(1 + r) * kTileBytes)), "l"(tmb[r]), "r"(k0), "r"((int)n0), "r"(bar) : "memory");
+                                 ::"r"(smem_u32(st + (size_t)(1 + r) * kTileBytes)), "l"(tmb[P.wide ? 0 : r]), "r"(k0),
+                                   "r"((int)n0 + (P.wide ? r * kBN : 0)), "r"(bar) : "memory");
             }
         }
     } else if (warp == 1) {
@@ -162,8 +165,12 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         if (!done) s_timeout = 1;
         const float sx = (m < P.M) ? P.sx[m] : 0.f;
         for (int r = 0; r < P.n_r; ++r) {
-            const float scale = (float)(1 << P.sh[r]);
-            float* yrow = P.Y[r] + m * P.ldy + n0;
+            const int pr = P.wide ? 0 : r;                    // which precision this accumulator belongs to
+            const int64_t nb = n0 + (P.wide ? r * kBN : 0);     // first channel of this accumulator
+            const float* al = s_alpha + (P.wide ? r * kBN : 0);
+            const float* az = s_az + (P.wide ? r * kBN : 0);
+            const float scale = (float)(1 << P.sh[pr]);
+            float* yrow = P.Y[pr] + m * P.ldy + nb;
             for (int c0 = 0; c0 < kBN; c0 += 32) {
                 uint32_t d[32];
                 const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + r * kBN + c0;
@@ -176,22 +183,22 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                              : "r"(addr) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (m < P.M) {
-                    const bool vec = (n0 + c0 + 32 <= P.N) && ((reinterpret_cast<uintptr_t>(yrow + c0) & 15u) == 0);
+                    const bool vec = (nb + c0 + 32 <= P.N) && ((reinterpret_cast<uintptr_t>(yrow + c0) & 15u) == 0);
                     if (vec) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 o;
-                            o.x = s_alpha[c0 + j] * scale * __uint_as_float(d[j]) - s_az[c0 + j] * sx;
-                            o.y = s_alpha[c0 + j + 1] * scale * __uint_as_float(d[j + 1]) - s_az[c0 + j + 1] * sx;
-                            o.z = s_alpha[c0 + j + 2] * scale * __uint_as_float(d[j + 2]) - s_az[c0 + j + 2] * sx;
-                            o.w = s_alpha[c0 + j + 3] * scale * __uint_as_float(d[j + 3]) - s_az[c0 + j + 3] * sx;
+                            o.x = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx;
+                            o.y = al[c0 + j + 1] * scale * __uint_as_float(d[j + 1]) - az[c0 + j + 1] * sx;
+                            o.z = al[c0 + j + 2] * scale * __uint_as_float(d[j + 2]) - az[c0 + j + 2] * sx;
+                            o.w = al[c0 + j + 3] * scale * __uint_as_float(d[j + 3]) - az[c0 + j + 3] * sx;
                             *reinterpret_cast<float4*>(yrow + c0 + j) = o;
                         }
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (n0 + c0 + j < P.N)
-                                yrow[c0 + j] = s_alpha[c0 + j] * scale * __uint_as_float(d[j]) - s_az[c0 + j] * sx;
+                            if (nb + c0 + j < P.N)
+                                yrow[c0 + j] = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx;
                     }
                 }
             }
@@ -454,6 +461,11 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
     for (int i = 0; i < kMaxR; ++i) { P.Y[i] = Y[i < n_r ? i : 0]; P.sh[i] = c - rs[i < n_r ? i : 0]; }
     P.M = M; P.N = N; P.K = K; P.ldy = ldy; P.n_r = n_r;
     P.dev_status = dev_status;
+    // A single plane would leave every MMA at N = 128 (shared-memory bound); the CTA then takes 256 channels as two
+    // adjacent tiles of the same plane so that one N = 256 instruction covers them.
+    P.wide = (n_r == 1 && N > kBN) ? 1 : 0;
+    if (P.wide) { P.n_r = 2; tm_b[1] = tm_b[0]; n_r = 2; }
+    const int cta_n = P.wide ? 2 * kBN : kBN;
     const int stage_bytes = (1 + n_r) * kTileBytes;
     int stages = (200 * 1024) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -461,7 +473,7 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     if (cudaFuncSetAttribute(gemm_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
-    const dim3 grid((unsigned)((M + kBM - 1) / kBM), (unsigned)((N + kBN - 1) / kBN), 1);
+    const dim3 grid((unsigned)((M + kBM - 1) / kBM), (unsigned)((N + cta_n - 1) / cta_n), 1);
     gemm_multi_kernel<<<grid, kThreads, smem, s>>>(tm_x, tm_b[0], tm_b[1], tm_b[2], P);
     return launch_status();
 }
