@@ -72,6 +72,21 @@ def test_packed_source(r, ep):
     assert torch.equal(Yc[0], Ys[0])
 
 
+@pytest.mark.parametrize("M,N,K", [(130, 128, 128), (130, 256, 192), (257, 392, 256), (64, 1000, 128), (300, 2056, 64), (33, 136, 64)])
+@pytest.mark.parametrize("r,ep", [(4, False), (2, True)])
+def test_single_precision_uses_256_channel_tiles(M, N, K, r, ep):
+    # one plane only: the CTA takes 256 channels (two adjacent tiles, one N = 256 MMA); ragged N in either half
+    W = synth.normal_bf16((N, K), 0.02, 70 + N)
+    st, q, a, z = ref.quantize(W)
+    if ep:
+        q = synth.skewed_codes((N, K), 0.05, 224, 71 + N)
+    X = synth.normal_bf16((M, K), 1.0, 72 + M)
+    Ys, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(r,), alpha=dev(a), zero=dev(z), extra_precision=ep)
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, q, K, X, rs=(r,), alpha=a, zero=z, extra_precision=ep)
+    assert st == ref.OK
+    _check(Ys, Yr)
+
+
 def test_exact_integer_case_and_independence_of_outputs():
     # alpha = 1, z = 0, integer activations: every partial sum is an exact fp32 integer
     M, N, K = 128, 128, 512
