@@ -421,9 +421,15 @@ def gemm_cfg4(mq, torch, peaks, reps=5):
 def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
     """configs[2] shapes: Gemma-2-9B decoder layers (q, k, v, o, gate, up, down), B = 1, r = 4 and r = 2.  The planes are
     random bytes (the kernels' speed does not depend on the field values); every matrix has its own buffers."""
-    shapes = [(n, k) for _ in range(layers) for (_, n, k) in synth.gemma2_9b_decoder_layer()]
-    out = {"workload": f"configs[2] Gemma-2-9B decoder layer shapes x {layers} layers, B = 1, one CUDA graph per precision, PDL"}
-    for r in (4, 2):
+    per_layer = [(n, k) for (_, n, k) in synth.gemma2_9b_decoder_layer()]
+    # q, k, v share their input and so do gate, up: stacked along N they are one matrix each (rows are quantised
+    # independently, so stacking changes no result); 4 launches per layer instead of 7
+    d, ff = per_layer[0][1], per_layer[4][0]
+    fused_layer = [(per_layer[0][0] + per_layer[1][0] + per_layer[2][0], d), per_layer[3], (2 * ff, d), per_layer[6]]
+    out = {"workload": f"configs[2] Gemma-2-9B decoder layer shapes x {layers} layers, B = 1, one CUDA graph per precision, PDL; "
+                       "'_fused' = q,k,v and gate,up stacked into one matrix each (4 launches per layer)"}
+    for r, fused in ((4, False), (2, False), (4, True), (2, True)):
+        shapes = [s for _ in range(layers) for s in (fused_layer if fused else per_layer)]
         planes = [torch.randint(0, 256, (n, k * r // 8), dtype=torch.uint8, device="cuda") for n, k in shapes]
         xs = [torch.randn(1, k, device="cuda").to(torch.bfloat16) for n, k in shapes]
         ys = [torch.empty(1, n, device="cuda") for n, k in shapes]
@@ -450,7 +456,7 @@ def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
         nbytes = sum(bytes_gemv(n, k, r, 1) for n, k in shapes)
-        out[f"r{r}_b1"] = {"ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
+        out[f"r{r}_b1" + ("_fused" if fused else "")] = {"ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
                            "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4), "launches": len(shapes)}
         del planes, xs, ys, al, g
         torch.cuda.empty_cache()
