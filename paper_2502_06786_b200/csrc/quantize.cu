@@ -232,12 +232,12 @@ quantize_rows_vec(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
     }
 }
 
-// Range of two bf16 values at a time: packed min / max (NaN operands are ignored, as fminf / fmaxf do) and a packed
-// "exponent all ones" detector: |v| + 0x0080 carries into bit 15 exactly when |v| >= 0x7f80 (Inf or NaN).
-__device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& mx2, uint32_t& bad2) {
-    asm("min.bf16x2 %0, %0, %1;" : "+r"(mn2) : "r"(w));
-    asm("max.bf16x2 %0, %0, %1;" : "+r"(mx2) : "r"(w));
-    bad2 |= (w & 0x7fff7fffu) + 0x00800080u;
+// Range of two bf16 values at a time: packed min / max that PROPAGATE NaN, so a NaN anywhere ends up in the running
+// pair and an Inf is the extreme itself: non-finite weights are detected once per thread from the four folded
+// values instead of once per weight.
+__device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& mx2) {
+    asm("min.NaN.bf16x2 %0, %0, %1;" : "+r"(mn2) : "r"(w));
+    asm("max.NaN.bf16x2 %0, %0, %1;" : "+r"(mx2) : "r"(w));
 }
 
 // Register-resident path (K <= 16384, K % 8 == 0): a team of 32 * WPR threads owns a row and keeps it in registers
@@ -259,7 +259,7 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
         const int64_t n = n_base + team;
         const bool live = n < N;
         uint4 v[NV];
-        uint32_t mn2 = 0x7f807f80u, mx2 = 0xff80ff80u, bad2 = 0;      // +Inf / -Inf pairs
+        uint32_t mn2 = 0x7f807f80u, mx2 = 0xff80ff80u;                // +Inf / -Inf pairs
         if (live) {
             const uint4* src = reinterpret_cast<const uint4*>(W + n * ldw);
 #pragma unroll
@@ -271,16 +271,19 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
             for (int j = 0; j < NV; ++j) {
                 const int i = team_tid + j * team_threads;
                 if (i < nvec) {
-                    fold_word2(v[j].x, mn2, mx2, bad2);
-                    fold_word2(v[j].y, mn2, mx2, bad2);
-                    fold_word2(v[j].z, mn2, mx2, bad2);
-                    fold_word2(v[j].w, mn2, mx2, bad2);
+                    fold_word2(v[j].x, mn2, mx2);
+                    fold_word2(v[j].y, mn2, mx2);
+                    fold_word2(v[j].z, mn2, mx2);
+                    fold_word2(v[j].w, mn2, mx2);
                 }
             }
         }
-        float mn = fminf(__uint_as_float(mn2 << 16), __uint_as_float(mn2 & 0xffff0000u));
-        float mx = fmaxf(__uint_as_float(mx2 << 16), __uint_as_float(mx2 & 0xffff0000u));
-        int bad = (bad2 & 0x80008000u) != 0;
+        // a thread that folded at least one piece (team_tid < nvec) sees +-Inf or NaN here only from a weight
+        const float mn_a = __uint_as_float(mn2 << 16), mn_b = __uint_as_float(mn2 & 0xffff0000u);
+        const float mx_a = __uint_as_float(mx2 << 16), mx_b = __uint_as_float(mx2 & 0xffff0000u);
+        float mn = fminf(mn_a, mn_b);
+        float mx = fmaxf(mx_a, mx_b);
+        int bad = live && team_tid < nvec && (!(fabsf(mn_a) <= 3.4e38f) | !(fabsf(mn_b) <= 3.4e38f) | !(fabsf(mx_a) <= 3.4e38f) | !(fabsf(mx_b) <= 3.4e38f));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
