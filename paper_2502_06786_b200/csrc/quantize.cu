@@ -244,7 +244,7 @@ __device__ __forceinline__ void fold_word2(uint32_t w, uint32_t& mn2, uint32_t& 
 // (NV 16-byte pieces per thread), so the row is read once, never touches shared memory, and every thread both
 // folds the range and emits codes.  A CTA of 8 warps works on 8 / WPR rows at a time.
 template <int NV, int WARPS, bool CLIP>
-__global__ void __launch_bounds__(WARPS * 32, (NV <= 5 ? 32 : 16) / WARPS)
+__global__ void __launch_bounds__(WARPS * 32, (NV <= 5 ? 32 : NV <= 9 ? 24 : 16) / WARPS)
 quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw, int wpr,
                   const float* __restrict__ gamma, const float* __restrict__ beta,
                   uint8_t* __restrict__ q, float* __restrict__ alpha, float* __restrict__ zero,
@@ -390,7 +390,7 @@ extern "C" int matq_quantize_clip(const void* W, int64_t N, int64_t K, int64_t l
     if (reg) {
         const int nvec = (int)(K / 8);
         int wpr = 1;
-        while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 5) wpr *= 2;
+        while (wpr < 8 && (nvec + 32 * wpr - 1) / (32 * wpr) > 9) wpr *= 2;
         const int nv = (nvec + 32 * wpr - 1) / (32 * wpr);
         // CTAs of 4 warps when a row's team fits (measured 5 % faster than 8: more CTAs per SM in different phases)
         const int warps = wpr <= 4 ? 4 : 8;
@@ -409,7 +409,8 @@ extern "C" int matq_quantize_clip(const void* W, int64_t N, int64_t K, int64_t l
         else if (nv <= 3) MATQ_QUANT_REG(3);
         else if (nv <= 4) MATQ_QUANT_REG(4);
         else if (nv <= 5) MATQ_QUANT_REG(5);
-        else MATQ_QUANT_REG(8);
+        else if (nv <= 7) MATQ_QUANT_REG(7);
+        else MATQ_QUANT_REG(9);
 #undef MATQ_QUANT_REG
     } else if (fast) {
         const size_t smem = (size_t)K * 2;
