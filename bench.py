@@ -364,6 +364,8 @@ def run_cuda(args, rank, world, local_rank):
         extras = {"gemv_cfg3": gemv_cfg3(mq, torch, peaks), "gemm_multi_cfg5_prefill": gemm_cfg5_prefill(mq, torch, peaks)}
         torch.cuda.empty_cache()
         extras["quantize_clip_cfg5"] = quantize_clip_cfg5(mq, torch, peaks)
+        torch.cuda.empty_cache()
+        extras["gemv_cfg2_mixnmatch"] = gemv_cfg2_mixnmatch(mq, torch, peaks)
 
     out = None
     if rank == 0:
@@ -499,6 +501,44 @@ def quantize_clip_cfg5(mq, torch, peaks, layers=2, reps=10):
     return {"workload": f"Eq. 3 on configs[4] weights: {layers} Gemma-2-9B MLP layers, Student-t(3), gamma = beta = 0.5, matq_quantize_clip",
             "ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1), "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4),
             "launches": len(shapes), "overflow_fraction_r2": round(int(sp["ovf_count"].item()) / (n0 * k0), 4)}
+
+
+def gemv_cfg2_mixnmatch(mq, torch, peaks, reps=10):
+    """Layer-wise Mix'n'Match on configs[1]: the 26-layer Gemma-2-2B MLP stack served with the Pyramid assignment
+    (int2 at both ends, int8 in the centre, int4 in between; 8 + 10 + 8 layers = 4.62 effective bits), B = 1, every
+    matrix of a layer at that layer's precision, one CUDA graph, PDL.  Planes are random bytes."""
+    from paper_2502_06786_b200 import mixnmatch
+    rs = mixnmatch.assign(8, 10, 8, "pyramid")
+    mats = [(n, k, rs[l]) for l in range(len(rs)) for (_, n, k) in synth.gemma2_2b_mlp_layer()]
+    planes = [torch.randint(0, 256, (n, k * r // 8), dtype=torch.uint8, device="cuda") for n, k, r in mats]
+    xs = [torch.randn(1, k, device="cuda").to(torch.bfloat16) for n, k, r in mats]
+    ys = [torch.empty(1, n, device="cuda") for n, k, r in mats]
+    al = [torch.ones(n, device="cuda") for n, k, r in mats]
+
+    def run():
+        for i, (n, k, r) in enumerate(mats):
+            mq.gemv(planes[i], k, r, al[i], al[i], xs[i], y=ys[i], flags=mq.GEMV_AUTO | mq.GEMV_PDL)
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            run()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    nbytes = sum(bytes_gemv(n, k, r, 1) for n, k, r in mats)
+    return {"workload": "configs[1] stack, Pyramid Mix'n'Match: 4 int2 + 5 int4 + 8 int8 + 5 int4 + 4 int2 layers, B = 1, PDL",
+            "effective_bits": round(mixnmatch.effective_bits(rs), 3), "ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
+            "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4), "launches": len(mats)}
 
 
 def gemm_cfg5_prefill(mq, torch, peaks, reps=3):
