@@ -45,7 +45,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     // (a second, partly filled wave costs up to 40 %; measured on B200 for 4-26 MB planes):
     //   * few, long rows (at most one or two 16-row tiles per SM): one tile per CTA of 32 or 16 warps, SK = 32 / 16;
     //   * otherwise CTAs of 8 warps with two m-tiles per warp (the staged activations are reused twice; two such
-    //     CTAs fit an SM) and the finest K split (8, else 4) that still fits one wave; if neither does, SK = 8 and
+    //     CTAs fit an SM) and the finest K split (8, 4, 2 or 1) that still fits one wave; if none does, SK = 8 and
     //     several waves.
     const int sms = sm_count();
     const int64_t n_qc = (K * r / 8 + 63) / 64;
@@ -58,8 +58,9 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     } else {
         mt = 2;
         const int64_t tiles32 = (N + 31) / 32;
-        sk = 8;
-        if (tiles32 > 2 * sms && (tiles32 + 1) / 2 <= 2 * sms && n_qc >= 4) sk = 4;
+        sk = 8;                                          // CTAs = tiles32 / (8 / sk): halve sk until they fit one wave
+        while (sk > 1 && (tiles32 * sk + 7) / 8 > 2 * sms) sk /= 2;
+        if ((tiles32 * sk + 7) / 8 > 2 * sms) sk = 8;     // not even SK = 1 fits: several waves of the finest split
         while (sk > 1 && n_qc < sk) sk /= 2;
     }
     int st;

@@ -266,7 +266,7 @@ def test_gemv_tcgen05_within_tolerance(r, N, K, B):
 @pytest.mark.parametrize("r", [4, 2])
 @pytest.mark.parametrize("N,K,B,ep", [(9216, 2304, 1, False), (9216, 2304, 8, False), (2304, 9216, 1, True), (14336, 3584, 1, False),
                                       (14336, 3584, 8, True), (4096, 3584, 2, False), (2048, 3584, 1, True), (3584, 14336, 8, False),
-                                      (9216, 2304, 1, True), (36864, 256, 3, False)])
+                                      (9216, 2304, 1, True), (36864, 256, 3, False), (75008, 128, 1, False), (151680, 128, 2, True)])
 def test_gemv_default_dispatch_at_benchmark_shapes(r, N, K, B, ep):
     # The library's own choice of warp tile, K split and CTA size (and the programmatic-dependent-launch flag the benchmark
     # passes) on the layer shapes of the Gemma-2-2B / 9B workloads, every output checked against the oracle.
