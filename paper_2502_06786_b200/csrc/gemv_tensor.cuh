@@ -462,7 +462,7 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     P.qc_pass = (P.n_qc + passes - 1) / passes;
     const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
     auto kern = ovf_row_ptr ? gemv_tensor<R, MT, NT, SK, WARPS, true> : gemv_tensor<R, MT, NT, SK, WARPS, false>;
-    if (smem > 48 * 1024 &&
+    if (smem > 16 * 1024 &&   // the 48 KB default counts static shared memory too
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};

@@ -506,7 +506,7 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     if (rpw < 1) return MATQ_ERR_SHAPE;
     const int T = nwarps * rpw;
     const size_t smem = (size_t)T * row_smem;
-    if (smem > 48 * 1024 &&
+    if (smem > 40 * 1024 &&   // the 48 KB default counts static shared memory too
         cudaFuncSetAttribute(slice_pack_ep<PACK_R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEpSmemLimit) != cudaSuccess)
         return MATQ_ERR_CUDA;
     int per_sm = 0;

@@ -274,6 +274,21 @@ def test_gemv_default_dispatch_at_benchmark_shapes(r, N, K, B, ep):
     assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
 
 
+def test_gemv_default_dispatch_on_random_shapes():
+    # Ragged N, every batch size class, short and long rows, with and without overflow lists: the split heuristic has
+    # many branches (SK = 1 .. 32, one or two m-tiles, 8 / 16 / 32 warps) and each must give the oracle's result.
+    rng = np.random.default_rng(2024)
+    for case in range(36):
+        N = int(rng.choice([1, 7, 16, 33, 100, 257, 600, 1500, 4100, 5000, 9500]))
+        K = 128 * int(rng.choice([1, 2, 3, 5, 8, 19, 36, 72]))
+        B = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16]))
+        r = int(rng.choice([8, 4, 2]))
+        ep = bool(rng.integers(0, 2)) and r < 8
+        y, y_ref = _gemv_case(N, K, B, r, 3000 + case, ep=ep, flags=mq.GEMV_AUTO | (mq.GEMV_PDL if case % 2 else 0))
+        assert y.shape == y_ref.shape
+        assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref), (N, K, B, r, ep)
+
+
 @pytest.mark.parametrize("flags,tol", [(mq.GEMV_CUDA_CORE, TOL_FMA), (mq.GEMV_TENSOR, TOL_TENSOR), (mq.GEMV_TCGEN05, TOL_TENSOR),
                                        (mq.GEMV_AUTO, TOL_TENSOR)])
 @pytest.mark.parametrize("r", [4, 2])
