@@ -167,3 +167,21 @@ def gemm_multi(src_kind: int, Wsrc: np.ndarray, K: int, X_bits: np.ndarray, rs=(
                                    _p(ovf_row_ptr), _p(ovf_col), _p(X_bits), C.c_int64(M), C.c_int64(K),
                                    rs_arr, C.c_int(len(rs)), Yp, C.c_int64(N), _p(qs), _p(S))
     return st, Ys, alpha, zero
+
+
+def gemm_multi_loss(src_kind: int, Wsrc: np.ndarray, K: int, X_bits: np.ndarray, Yt: np.ndarray, lambdas, rs=(8, 4, 2),
+                    alpha=None, zero=None, extra_precision: bool = False, ovf_row_ptr=None, ovf_col=None, c: int = 8):
+    """Eq. 7 with the L2 reconstruction loss of Eq. 5 for one linear layer: for every r in ``rs``
+    L_r = sum over tokens and channels of (Yt - F(S(Q(W, c), r), X))^2 against a given target Yt (fp32 [M, N], e.g. the
+    bf16 layer's output), and the weighted objective sum_r lambda_r L_r (no 1/N: the caller divides by its sample count).
+    The definition written out with NumPy in float64 on top of ``gemm_multi``.
+    Returns (status, [L_r], total, alpha, zero)."""
+    assert Yt.dtype == np.float32 and len(lambdas) == len(rs)
+    st, Ys, alpha, zero = gemm_multi(src_kind, Wsrc, K, X_bits, rs=rs, alpha=alpha, zero=zero,
+                                     extra_precision=extra_precision, ovf_row_ptr=ovf_row_ptr, ovf_col=ovf_col, c=c)
+    if st != OK:
+        return st, None, None, alpha, zero
+    t = Yt.astype(np.float64)
+    losses = [float(((t - y) ** 2).sum()) for y in Ys]
+    total = float(sum(float(l) * L for l, L in zip(lambdas, losses)))
+    return st, losses, total, alpha, zero
