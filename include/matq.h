@@ -188,6 +188,30 @@ int matq_gemm_multi(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
                     int32_t *dev_status, void *stream);
 
 /*
+ * (4b) The objective of MatQuant co-training for one linear layer (Eq. 7 with the L2 reconstruction loss of Eq. 5):
+ *       L_r   = sum_{m,n} ( Yt[m,n] - Y_r[m,n] )^2   for every r in rs, Y_r as in matq_gemm_multi,
+ *       total = sum_i lambda[i] * L_{rs[i]}
+ *     computed in the epilogue of the same tensor-core pass: the n_r outputs are compared with the target while they
+ *     are still in tensor memory and are never written to HBM (for R = {8, 4, 2} that is 12 bytes per output element
+ *     not stored).  No 1/N: the caller divides by its sample count.
+ *   lambda  in   HOST array of n_r loss weights (Eq. 7's lambda_r)
+ *   Yt      in   fp32 [M, N] target, row stride ldt elements (e.g. the bf16 layer's output F(W_F, X))
+ *   loss    out  DEVICE double [n_r + 1]: L_{rs[0]}, ..., L_{rs[n_r-1]}, total.  Per-thread and per-CTA sums are fp32,
+ *                the sum over CTAs is double, all in a fixed order: results are reproducible run to run.
+ *   workspace    at least matq_gemm_multi_loss_workspace_bytes(...) bytes, 256-byte aligned
+ *   Everything else as for matq_gemm_multi.
+ */
+size_t matq_gemm_multi_loss_workspace_bytes(int src_kind, int64_t M, int64_t N, int64_t K, int n_r);
+int matq_gemm_multi_loss(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
+                         float *alpha, float *zero, int extra_precision,
+                         const int32_t *ovf_row_ptr, const uint16_t *ovf_col,
+                         const void *X, int64_t M, int64_t ldx,
+                         const int *rs, int n_r, const float *lambda,
+                         const float *Yt, int64_t ldt, double *loss,
+                         void *workspace, size_t workspace_bytes,
+                         int32_t *dev_status, void *stream);
+
+/*
  * (5) matq_gemm_multi without a workspace argument.  The paper has no counterpart to this call: it exists for
  *     callers that cannot obtain device memory when they call the library (a serving loop whose memory was divided
  *     up at start-up and that must not call cudaMalloc on the request path, because that call synchronises the

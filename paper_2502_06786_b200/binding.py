@@ -24,6 +24,7 @@ GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_PDL = 0, 1, 2, 3, 0x1
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
            "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
+           "matq_gemm_multi_loss_workspace_bytes", "matq_gemm_multi_loss",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
 
 
@@ -60,6 +61,11 @@ def _load():
     lib.matq_gemm_multi.restype = i32
     lib.matq_gemm_multi.argtypes = [i32, vp, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, i64,
                                     C.POINTER(C.c_int), i32, C.POINTER(C.c_void_p), i64, vp, sz, vp, vp]
+    lib.matq_gemm_multi_loss_workspace_bytes.restype = sz
+    lib.matq_gemm_multi_loss_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
+    lib.matq_gemm_multi_loss.restype = i32
+    lib.matq_gemm_multi_loss.argtypes = [i32, vp, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, i64,
+                                         C.POINTER(C.c_int), i32, C.POINTER(C.c_float), vp, i64, vp, vp, sz, vp, vp]
     lib.matq_gemm_multi_static_max_bytes.restype = sz
     lib.matq_gemm_multi_static_max_bytes.argtypes = []
     lib.matq_gemm_multi_static.restype = i32
@@ -231,6 +237,43 @@ def gemm_multi(src_kind, Wsrc, K, X, rs=(8, 4, 2), alpha=None, zero=None, extra_
                               workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream())
     _check(st, "matq_gemm_multi")
     return Ys, alpha, zero
+
+
+def gemm_multi_loss_workspace_bytes(src_kind, M, N, K, n_r) -> int:
+    return int(_lib.matq_gemm_multi_loss_workspace_bytes(src_kind, M, N, K, n_r))
+
+
+def gemm_multi_loss(src_kind, Wsrc, K, X, Yt, lambdas, rs=(8, 4, 2), alpha=None, zero=None, extra_precision=False,
+                    ovf_row_ptr=None, ovf_col=None, loss=None, workspace=None, dev_status=None, c=8):
+    """matq_gemm_multi_loss.  Yt: fp32 [M, N] target.  Returns (loss, alpha, zero); loss is a device float64 tensor
+    [len(rs) + 1]: one squared error per precision and the lambda-weighted total."""
+    _dev(X, torch.bfloat16, "X", 2)
+    _dev(Yt, torch.float32, "Yt", 2)
+    _dev(Wsrc, torch.bfloat16 if src_kind == SRC_BF16 else torch.uint8, "Wsrc", 2)
+    if len(lambdas) != len(rs):
+        raise ValueError("one lambda per precision")
+    N = Wsrc.shape[0]
+    M = X.shape[0]
+    dev = X.device
+    if Yt.shape != (M, N) or Yt.stride(1) != 1:
+        raise ValueError("Yt: fp32 [M, N] with unit stride along N required")
+    if alpha is None:
+        alpha = torch.empty(N, dtype=torch.float32, device=dev)
+    if zero is None:
+        zero = torch.empty(N, dtype=torch.float32, device=dev)
+    if loss is None:
+        loss = torch.empty(len(rs) + 1, dtype=torch.float64, device=dev)
+    need = gemm_multi_loss_workspace_bytes(src_kind, M, N, K, len(rs))
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    rs_arr = (C.c_int * len(rs))(*rs)
+    lam = (C.c_float * len(rs))(*[float(v) for v in lambdas])
+    st = _lib.matq_gemm_multi_loss(src_kind, _ptr(Wsrc), N, K, c, _ptr(alpha), _ptr(zero), int(bool(extra_precision)),
+                                   _ptr(ovf_row_ptr), _ptr(ovf_col), _ptr(X), M, _ld(X, K), rs_arr, len(rs), lam,
+                                   _ptr(Yt), _ld(Yt, N), _ptr(loss), _ptr(workspace),
+                                   workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream())
+    _check(st, "matq_gemm_multi_loss")
+    return loss, alpha, zero
 
 
 def gemm_multi_static_max_bytes() -> int:

@@ -39,6 +39,9 @@ struct Params {
     int64_t M, N, K, ldy;
     int n_r, stages;
     int wide;      // one plane only: the CTA takes 256 channels as two adjacent 128-row tiles (n_r is then 2)
+    const float* Yt;      // loss mode: target [M, N] (row stride ldt); outputs are not stored
+    int64_t ldt;
+    float* loss_part;     // loss mode: [CTAs][kMaxR] sums of squared errors
     int32_t* dev_status;
 };
 
@@ -69,6 +72,7 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     __shared__ uint32_t s_tmem;
     __shared__ float s_alpha[2 * kBN], s_az[2 * kBN];      // alpha_n and alpha_n * z_n of this tile's columns
     __shared__ int s_timeout;
+    __shared__ float s_loss[4][kMaxR];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // blockIdx.x walks the token tiles: CTAs that run together share one 128-channel slab of the planes (3 x 1 MB,
@@ -164,15 +168,24 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (!done) s_timeout = 1;
         const float sx = (m < P.M) ? P.sx[m] : 0.f;
+        float lacc[kMaxR] = {0.f, 0.f, 0.f};               // loss mode: this thread's squared errors per precision
         for (int r = 0; r < P.n_r; ++r) {
             const int pr = P.wide ? 0 : r;                    // which precision this accumulator belongs to
             const int64_t nb = n0 + (P.wide ? r * kBN : 0);     // first channel of this accumulator
             const float* al = s_alpha + (P.wide ? r * kBN : 0);
             const float* az = s_az + (P.wide ? r * kBN : 0);
             const float scale = (float)(1 << P.sh[pr]);
-            float* yrow = P.Y[pr] + m * P.ldy + nb;
+            float* yrow = P.Yt ? nullptr : P.Y[pr] + m * P.ldy + nb;
             for (int c0 = 0; c0 < kBN; c0 += 32) {
                 uint32_t d[32];
+                // loss mode: the thread's 128 bytes of the target row are requested before the accumulators are read
+                const float* trow = P.Yt ? P.Yt + m * P.ldt + nb + c0 : nullptr;
+                const bool tvec = P.Yt && m < P.M && (nb + c0 + 32 <= P.N) && ((reinterpret_cast<uintptr_t>(trow) & 15u) == 0);
+                float4 t4[8];
+                if (tvec) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) t4[j] = __ldg(reinterpret_cast<const float4*>(trow) + j);
+                }
                 const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + r * kBN + c0;
                 asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                              "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -182,7 +195,31 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                                "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
                              : "r"(addr) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (m < P.M) {
+                if (P.Yt) {                                   // Eq. 7's loss against the target instead of the outputs
+                    if (m < P.M) {
+                        float acc = 0.f;
+                        if (tvec) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float tv[4] = {t4[j].x, t4[j].y, t4[j].z, t4[j].w};
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int cc = c0 + 4 * j + u;
+                                    const float e = al[cc] * scale * __uint_as_float(d[4 * j + u]) - az[cc] * sx - tv[u];
+                                    acc = fmaf(e, e, acc);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + c0 + j < P.N) {
+                                    const float e = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx - trow[j];
+                                    acc = fmaf(e, e, acc);
+                                }
+                        }
+                        lacc[pr] += acc;
+                    }
+                } else if (m < P.M) {
                     const bool vec = (nb + c0 + 32 <= P.N) && ((reinterpret_cast<uintptr_t>(yrow + c0) & 15u) == 0);
                     if (vec) {
 #pragma unroll
@@ -203,9 +240,21 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 }
             }
         }
+        if (P.Yt) {                                           // warp sums in a fixed order, one slot per epilogue warp
+#pragma unroll
+            for (int i = 0; i < kMaxR; ++i) {
+                float v = lacc[i];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) s_loss[quad][i] = v;
+            }
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (P.Yt && tid < kMaxR)
+        P.loss_part[((size_t)blockIdx.y * gridDim.x + blockIdx.x) * kMaxR + tid] =
+            (s_loss[0][tid] + s_loss[1][tid]) + (s_loss[2][tid] + s_loss[3][tid]);
     if (tid == 0 && s_timeout) report(P.dev_status, MATQ_ERR_TIMEOUT);
     if (warp == 2)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols) : "memory");
@@ -347,6 +396,30 @@ struct Layout {
     size_t codes_off, plane_off, plane_bytes, sx_off, total;
 };
 
+// Sums the per-CTA squared errors in double precision and in a fixed order: thread t adds the CTAs t, t + 256, ...
+// and the 256 thread sums are folded by a tree.  loss[i] = L_{rs[i]}, loss[n_r] = sum_i lambda_i L_i.
+struct LossArgs {
+    float lambda[kMaxR];
+    int n_r;
+};
+__global__ void __launch_bounds__(256) loss_reduce(const float* __restrict__ part, int64_t n_cta, LossArgs A, double* __restrict__ loss) {
+    __shared__ double s[256];
+    double total = 0.0;
+    for (int i = 0; i < A.n_r; ++i) {
+        double v = 0.0;
+        for (int64_t c = threadIdx.x; c < n_cta; c += 256) v += (double)part[c * kMaxR + i];
+        s[threadIdx.x] = v;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if ((int)threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) { loss[i] = s[0]; total += (double)A.lambda[i] * s[0]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) loss[A.n_r] = total;
+}
+
 inline Layout layout(int src_kind, int64_t M, int64_t N, int64_t K, int n_r) {
     Layout L;
     size_t off = 0;
@@ -370,16 +443,29 @@ extern "C" size_t matq_gemm_multi_workspace_bytes(int src_kind, int64_t M, int64
     return matq::gm::layout(src_kind, M, N, K, n_r).total;
 }
 
-extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_t K, int c,
-                               float* alpha, float* zero, int extra_precision,
-                               const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
-                               const void* X, int64_t M, int64_t ldx,
-                               const int* rs, int n_r, float* const* Y, int64_t ldy,
-                               void* workspace, size_t workspace_bytes,
-                               int32_t* dev_status, void* stream) {
+namespace matq {
+namespace gm {
+// Loss partials live behind the forward's workspace, 256-byte aligned.
+inline size_t loss_part_off(const Layout& L) { return (L.total + 255) / 256 * 256; }
+inline int64_t cta_count(int64_t M, int64_t N, int n_r) {
+    const int64_t cta_n = (n_r == 1 && N > kBN) ? 2 * kBN : kBN;
+    return ((M + kBM - 1) / kBM) * ((N + cta_n - 1) / cta_n);
+}
+}  // namespace gm
+}  // namespace matq
+
+// The forward (Y != NULL, Yt == NULL) or the loss (Yt != NULL, loss_part != NULL; nothing is stored to Y).
+static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K, int c,
+                           float* alpha, float* zero, int extra_precision,
+                           const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
+                           const void* X, int64_t M, int64_t ldx,
+                           const int* rs, int n_r, float* const* Y, int64_t ldy,
+                           const float* Yt, int64_t ldt, float* loss_part,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* dev_status, void* stream) {
     using namespace matq;
     using namespace matq::gm;
-    if (M < 0 || N < 0 || K <= 0 || !rs || !Y || n_r < 1 || n_r > kMaxR) return MATQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K <= 0 || !rs || (!Y && !Yt) || n_r < 1 || n_r > kMaxR) return MATQ_ERR_INVALID_ARG;
     if (src_kind < MATQ_SRC_BF16 || src_kind > MATQ_SRC_PACKED) return MATQ_ERR_INVALID_ARG;
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     for (int i = 0; i < n_r; ++i) {
@@ -391,10 +477,10 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
         if (!(rs[0] == 8 || rs[0] == 4 || rs[0] == 2)) return MATQ_ERR_UNSUPPORTED;
         if ((ovf_row_ptr == nullptr) != (ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
     }
-    if (K % kBK != 0 || N % 8 != 0 || ldx < K || ldx % 8 != 0 || ldy < N) return MATQ_ERR_SHAPE;
+    if (K % kBK != 0 || N % 8 != 0 || ldx < K || ldx % 8 != 0 || (Y && ldy < N) || (Yt && ldt < N)) return MATQ_ERR_SHAPE;
     if (M == 0 || N == 0) return MATQ_OK;
     if (!Wsrc || !alpha || !zero || !X) return MATQ_ERR_INVALID_ARG;
-    for (int i = 0; i < n_r; ++i) if (!Y[i]) return MATQ_ERR_INVALID_ARG;
+    if (Y) for (int i = 0; i < n_r; ++i) if (!Y[i]) return MATQ_ERR_INVALID_ARG;
     if (!aligned16(Wsrc) || !aligned16(X)) return MATQ_ERR_ALIGNMENT;
     const Layout L = layout(src_kind, M, N, K, n_r);
     if (!workspace || workspace_bytes < L.total) return MATQ_ERR_WORKSPACE;
@@ -458,7 +544,8 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
         if (!make_map(&tm_b[i], EA.plane[i], N, K, K)) return MATQ_ERR_CUDA;
     Params P;
     P.alpha = alpha; P.zero = zero; P.sx = sx;
-    for (int i = 0; i < kMaxR; ++i) { P.Y[i] = Y[i < n_r ? i : 0]; P.sh[i] = c - rs[i < n_r ? i : 0]; }
+    for (int i = 0; i < kMaxR; ++i) { P.Y[i] = Y ? Y[i < n_r ? i : 0] : nullptr; P.sh[i] = c - rs[i < n_r ? i : 0]; }
+    P.Yt = Yt; P.ldt = ldt; P.loss_part = loss_part;
     P.M = M; P.N = N; P.K = K; P.ldy = ldy; P.n_r = n_r;
     P.dev_status = dev_status;
     // A single plane would leave every MMA at N = 128 (shared-memory bound); the CTA then takes 256 channels as two
@@ -475,5 +562,53 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
         return MATQ_ERR_CUDA;
     const dim3 grid((unsigned)((M + kBM - 1) / kBM), (unsigned)((N + cta_n - 1) / cta_n), 1);
     gemm_multi_kernel<<<grid, kThreads, smem, s>>>(tm_x, tm_b[0], tm_b[1], tm_b[2], P);
+    return launch_status();
+}
+
+extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_t K, int c,
+                               float* alpha, float* zero, int extra_precision,
+                               const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
+                               const void* X, int64_t M, int64_t ldx,
+                               const int* rs, int n_r, float* const* Y, int64_t ldy,
+                               void* workspace, size_t workspace_bytes,
+                               int32_t* dev_status, void* stream) {
+    if (!Y) return MATQ_ERR_INVALID_ARG;
+    return gemm_multi_impl(src_kind, Wsrc, N, K, c, alpha, zero, extra_precision, ovf_row_ptr, ovf_col, X, M, ldx, rs, n_r,
+                           Y, ldy, nullptr, 0, nullptr, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" size_t matq_gemm_multi_loss_workspace_bytes(int src_kind, int64_t M, int64_t N, int64_t K, int n_r) {
+    using namespace matq::gm;
+    if (M < 0 || N < 0 || K <= 0 || n_r < 1 || n_r > kMaxR || src_kind < MATQ_SRC_BF16 || src_kind > MATQ_SRC_PACKED)
+        return 0;
+    return loss_part_off(layout(src_kind, M, N, K, n_r)) + (size_t)cta_count(M, N, n_r) * kMaxR * sizeof(float);
+}
+
+extern "C" int matq_gemm_multi_loss(int src_kind, const void* Wsrc, int64_t N, int64_t K, int c,
+                                    float* alpha, float* zero, int extra_precision,
+                                    const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
+                                    const void* X, int64_t M, int64_t ldx,
+                                    const int* rs, int n_r, const float* lambda,
+                                    const float* Yt, int64_t ldt, double* loss,
+                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* dev_status, void* stream) {
+    using namespace matq;
+    using namespace matq::gm;
+    if (!lambda || !loss || !Yt || n_r < 1 || n_r > kMaxR || M < 0 || N < 0 || K <= 0) return MATQ_ERR_INVALID_ARG;
+    if (src_kind < MATQ_SRC_BF16 || src_kind > MATQ_SRC_PACKED) return MATQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (M == 0 || N == 0)                                        // nothing to compare: every loss is zero
+        return cudaMemsetAsync(loss, 0, (size_t)(n_r + 1) * sizeof(double), s) == cudaSuccess ? MATQ_OK : MATQ_ERR_CUDA;
+    const size_t need = matq_gemm_multi_loss_workspace_bytes(src_kind, M, N, K, n_r);
+    if (!workspace || workspace_bytes < need) return MATQ_ERR_WORKSPACE;
+    const Layout L = layout(src_kind, M, N, K, n_r);
+    float* part = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + loss_part_off(L));
+    const int st = gemm_multi_impl(src_kind, Wsrc, N, K, c, alpha, zero, extra_precision, ovf_row_ptr, ovf_col, X, M, ldx,
+                                   rs, n_r, nullptr, 0, Yt, ldt, part, workspace, L.total, dev_status, stream);
+    if (st != MATQ_OK) return st;
+    LossArgs A;
+    A.n_r = n_r;
+    for (int i = 0; i < kMaxR; ++i) A.lambda[i] = i < n_r ? lambda[i] : 0.f;
+    loss_reduce<<<1, 256, 0, s>>>(part, cta_count(M, N, n_r), A, loss);
     return launch_status();
 }

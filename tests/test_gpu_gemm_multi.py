@@ -87,6 +87,48 @@ def test_single_precision_uses_256_channel_tiles(M, N, K, r, ep):
     _check(Ys, Yr)
 
 
+@pytest.mark.parametrize("M,N,K,rs", [(200, 264, 256, (8, 4, 2)), (130, 1000, 192, (8, 4, 2)), (64, 136, 128, (4,)),
+                                      (300, 520, 64, (2,)), (1, 8, 64, (8, 2)), (257, 392, 320, (6, 3))])
+def test_loss_matches_the_definition(M, N, K, rs):
+    # Eq. 7 with the L2 loss of Eq. 5: squared error of every precision against a target, in the GEMM's epilogue
+    W = synth.normal_bf16((N, K), 0.02, 80 + M)
+    X = synth.normal_bf16((M, K), 1.0, 81 + M)
+    Wf = synth.bf16_bits_to_f32(W).astype(np.float64)
+    Xf = synth.bf16_bits_to_f32(X).astype(np.float64)
+    Yt = (Xf @ Wf.T).astype(np.float32)                      # the unquantised layer's output
+    lam = tuple(0.5 + 0.75 * i for i in range(len(rs)))
+    st, L_ref, total_ref, a_ref, z_ref = ref.gemm_multi_loss(ref.SRC_BF16, W, K, X, Yt, lam, rs=rs)
+    assert st == ref.OK
+    status = status_word()
+    loss, a, z = mq.gemm_multi_loss(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), dev(Yt), lam, rs=rs, dev_status=status)
+    got = host(loss)
+    assert np.array_equal(host(a), a_ref) and np.array_equal(host(z), z_ref)
+    assert np.allclose(got[:-1], L_ref, rtol=2e-3) and np.isclose(got[-1], total_ref, rtol=2e-3), (got, L_ref)
+    assert int(host(status)[0]) == mq.OK
+    # reproducible bit for bit, and the forward's outputs give the same numbers when differenced on the host
+    loss2, _, _ = mq.gemm_multi_loss(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), dev(Yt), lam, rs=rs)
+    assert np.array_equal(host(loss2), got)
+    Ys, _, _ = mq.gemm_multi(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), rs=rs)
+    for i, y in enumerate(Ys):
+        want = float(((Yt.astype(np.float64) - host(y).astype(np.float64)) ** 2).sum())
+        assert np.isclose(got[i], want, rtol=1e-4)
+
+
+def test_loss_is_zero_against_its_own_int8_forward_in_the_integer_case():
+    rng = np.random.default_rng(9)
+    N, K, M = 136, 128, 70
+    q = rng.integers(0, 256, (N, K)).astype(np.uint8)
+    x = rng.integers(-3, 4, (M, K)).astype(np.float32)
+    one, zer = np.ones(N, np.float32), np.zeros(N, np.float32)
+    y8 = (x.astype(np.int64) @ q.astype(np.int64).T).astype(np.float32)
+    loss, _, _ = mq.gemm_multi_loss(mq.SRC_CODES8, dev(q), K, bf16_dev(synth.f32_to_bf16_bits(x)), dev(y8), (1.0, 1.0, 1.0),
+                                    alpha=dev(one), zero=dev(zer))
+    st, L_ref, total_ref, _, _ = ref.gemm_multi_loss(ref.SRC_CODES8, q, K, synth.f32_to_bf16_bits(x), y8, (1.0, 1.0, 1.0), alpha=one, zero=zer)
+    got = host(loss)
+    assert got[0] == 0.0 and L_ref[0] == 0.0
+    assert np.allclose(got[1:3], L_ref[1:], rtol=1e-5)
+
+
 def test_exact_integer_case_and_independence_of_outputs():
     # alpha = 1, z = 0, integer activations: every partial sum is an exact fp32 integer
     M, N, K = 128, 128, 512
