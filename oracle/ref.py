@@ -169,8 +169,12 @@ def gemm_multi(src_kind: int, Wsrc: np.ndarray, K: int, X_bits: np.ndarray, rs=(
     return st, Ys, alpha, zero
 
 
+TEACHER_AND_TARGET = 256
+
+
 def gemm_multi_loss(src_kind: int, Wsrc: np.ndarray, K: int, X_bits: np.ndarray, Yt: np.ndarray, lambdas, rs=(8, 4, 2),
-                    alpha=None, zero=None, extra_precision: bool = False, ovf_row_ptr=None, ovf_col=None, c: int = 8):
+                    alpha=None, zero=None, extra_precision: bool = False, ovf_row_ptr=None, ovf_col=None, c: int = 8,
+                    teacher=None):
     """Eq. 7 with the L2 reconstruction loss of Eq. 5 for one linear layer: for every r in ``rs``
     L_r = sum over tokens and channels of (Yt - F(S(Q(W, c), r), X))^2 against a given target Yt (fp32 [M, N], e.g. the
     bf16 layer's output), and the weighted objective sum_r lambda_r L_r (no 1/N: the caller divides by its sample count).
@@ -182,6 +186,16 @@ def gemm_multi_loss(src_kind: int, Wsrc: np.ndarray, K: int, X_bits: np.ndarray,
     if st != OK:
         return st, None, None, alpha, zero
     t = Yt.astype(np.float64)
-    losses = [float(((t - y) ** 2).sum()) for y in Ys]
+    losses = []
+    for i, y in enumerate(Ys):
+        # co-distillation (Section 5.2): teacher[i] = j >= 0 replaces the target of precision i by the output of the
+        # higher-precision nested model rs[j]; j + TEACHER_AND_TARGET uses both, weighted equally; -1 = target only
+        code = -1 if teacher is None else int(teacher[i])
+        L = 0.0
+        if code < 0 or code >= TEACHER_AND_TARGET:
+            L += float(((t - y) ** 2).sum())
+        if code >= 0:
+            L += float(((Ys[code % TEACHER_AND_TARGET] - y) ** 2).sum())
+        losses.append(L)
     total = float(sum(float(l) * L for l, L in zip(lambdas, losses)))
     return st, losses, total, alpha, zero

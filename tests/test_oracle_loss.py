@@ -56,3 +56,17 @@ def test_weights_are_linear_and_target_shift_is_quadratic():
     for r in range(3):
         resid = float((Yt.astype(np.float64) - Ys[r]).sum())
         assert np.isclose(L3[r], L[r] + Yt.size * d * d + 2 * d * resid, rtol=1e-5)      # Yt + d rounds in fp32
+
+
+def test_co_distillation_hand_values():
+    # the one-weight case again: Y_8 = 95, Y_4 = 99, Y_2 = 91, target 100.
+    q = np.array([[200]], np.uint8)
+    args = (ref.SRC_CODES8, q, 1, _bits([[1.0]]), np.array([[100.0]], np.float32), (1.0, 1.0, 1.0))
+    kw = dict(alpha=np.array([0.5], np.float32), zero=np.array([10.0], np.float32))
+    st, L, total, _, _ = ref.gemm_multi_loss(*args, teacher=(-1, 0, 0), **kw)          # int8 teaches int4 and int2
+    assert L == [25.0, 16.0, 16.0] and total == 57.0
+    st, L, total, _, _ = ref.gemm_multi_loss(*args, teacher=(-1, -1, 1), **kw)         # int4 teaches int2: (99 - 91)^2
+    assert L == [25.0, 1.0, 64.0]
+    both = ref.TEACHER_AND_TARGET
+    st, L, total, _, _ = ref.gemm_multi_loss(*args, teacher=(-1, -1, both + 0), **kw)  # target and int8 teacher, equal weights
+    assert L == [25.0, 1.0, 81.0 + 16.0]
