@@ -195,6 +195,9 @@ int matq_gemm_multi(int src_kind, const void *Wsrc, int64_t N, int64_t K, int c,
  *     are still in tensor memory and are never written to HBM (for R = {8, 4, 2} that is 12 bytes per output element
  *     not stored).  No 1/N: the caller divides by its sample count.
  *   lambda  in   HOST array of n_r loss weights (Eq. 7's lambda_r)
+ *   teacher in   HOST array of n_r ints or NULL (co-distillation, Section 5.2): -1 = precision i is compared with Yt;
+ *                j in [0, n_r), j != i = it is compared with Y_{rs[j]}, the output of that (higher-precision) nested
+ *                model, instead; 256 + j = with both, the two squared errors added.  NULL = all -1.
  *   Yt      in   fp32 [M, N] target, row stride ldt elements (e.g. the bf16 layer's output F(W_F, X))
  *   loss    out  DEVICE double [n_r + 1]: L_{rs[0]}, ..., L_{rs[n_r-1]}, total.  Per-thread and per-CTA sums are fp32,
  *                the sum over CTAs is double, all in a fixed order: results are reproducible run to run.
@@ -206,7 +209,7 @@ int matq_gemm_multi_loss(int src_kind, const void *Wsrc, int64_t N, int64_t K, i
                          float *alpha, float *zero, int extra_precision,
                          const int32_t *ovf_row_ptr, const uint16_t *ovf_col,
                          const void *X, int64_t M, int64_t ldx,
-                         const int *rs, int n_r, const float *lambda,
+                         const int *rs, int n_r, const float *lambda, const int *teacher,
                          const float *Yt, int64_t ldt, double *loss,
                          void *workspace, size_t workspace_bytes,
                          int32_t *dev_status, void *stream);

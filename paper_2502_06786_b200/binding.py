@@ -20,6 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_SHAPE, ERR_ALIGNMENT = 0, 1, 2, 3, 4
 ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_CAPACITY, ERR_TIMEOUT = 5, 6, 8, 9, 10
 SRC_BF16, SRC_CODES8, SRC_PACKED = 0, 1, 2
 GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_PDL = 0, 1, 2, 3, 0x100
+TEACHER_AND_TARGET = 256    # matq_gemm_multi_loss: teacher[i] = TEACHER_AND_TARGET + j
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
            "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv",
@@ -65,7 +66,7 @@ def _load():
     lib.matq_gemm_multi_loss_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
     lib.matq_gemm_multi_loss.restype = i32
     lib.matq_gemm_multi_loss.argtypes = [i32, vp, i64, i64, i32, vp, vp, i32, vp, vp, vp, i64, i64,
-                                         C.POINTER(C.c_int), i32, C.POINTER(C.c_float), vp, i64, vp, vp, sz, vp, vp]
+                                         C.POINTER(C.c_int), i32, C.POINTER(C.c_float), C.POINTER(C.c_int), vp, i64, vp, vp, sz, vp, vp]
     lib.matq_gemm_multi_static_max_bytes.restype = sz
     lib.matq_gemm_multi_static_max_bytes.argtypes = []
     lib.matq_gemm_multi_static.restype = i32
@@ -244,7 +245,7 @@ def gemm_multi_loss_workspace_bytes(src_kind, M, N, K, n_r) -> int:
 
 
 def gemm_multi_loss(src_kind, Wsrc, K, X, Yt, lambdas, rs=(8, 4, 2), alpha=None, zero=None, extra_precision=False,
-                    ovf_row_ptr=None, ovf_col=None, loss=None, workspace=None, dev_status=None, c=8):
+                    ovf_row_ptr=None, ovf_col=None, loss=None, workspace=None, dev_status=None, c=8, teacher=None):
     """matq_gemm_multi_loss.  Yt: fp32 [M, N] target.  Returns (loss, alpha, zero); loss is a device float64 tensor
     [len(rs) + 1]: one squared error per precision and the lambda-weighted total."""
     _dev(X, torch.bfloat16, "X", 2)
@@ -268,8 +269,9 @@ def gemm_multi_loss(src_kind, Wsrc, K, X, Yt, lambdas, rs=(8, 4, 2), alpha=None,
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
     rs_arr = (C.c_int * len(rs))(*rs)
     lam = (C.c_float * len(rs))(*[float(v) for v in lambdas])
+    tch = (C.c_int * len(rs))(*[int(v) for v in teacher]) if teacher is not None else None
     st = _lib.matq_gemm_multi_loss(src_kind, _ptr(Wsrc), N, K, c, _ptr(alpha), _ptr(zero), int(bool(extra_precision)),
-                                   _ptr(ovf_row_ptr), _ptr(ovf_col), _ptr(X), M, _ld(X, K), rs_arr, len(rs), lam,
+                                   _ptr(ovf_row_ptr), _ptr(ovf_col), _ptr(X), M, _ld(X, K), rs_arr, len(rs), lam, tch,
                                    _ptr(Yt), _ld(Yt, N), _ptr(loss), _ptr(workspace),
                                    workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream())
     _check(st, "matq_gemm_multi_loss")

@@ -42,6 +42,7 @@ struct Params {
     const float* Yt;      // loss mode: target [M, N] (row stride ldt); outputs are not stored
     int64_t ldt;
     float* loss_part;     // loss mode: [CTAs][kMaxR] sums of squared errors
+    int teacher[kMaxR];   // loss mode, per precision: -1 target only, j another precision's output as the target, 256 + j both
     int32_t* dev_status;
 };
 
@@ -58,6 +59,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 // K-major operand tile written by TMA with 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart.
 __device__ __forceinline__ uint64_t sw128_desc(uint32_t smem_addr) {
     return (uint64_t)((smem_addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&d)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
+                   "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
+                   "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
+                   "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
+                 : "r"(addr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 // kind::f16, D = fp32, A = B = bf16, both K-major, N = 128, M = 128
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
@@ -187,35 +199,32 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     for (int j = 0; j < 8; ++j) t4[j] = __ldg(reinterpret_cast<const float4*>(trow) + j);
                 }
                 const uint32_t addr = tmem + ((uint32_t)(quad * 32) << 16) + r * kBN + c0;
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                             "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                             : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
-                               "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15]),
-                               "=r"(d[16]), "=r"(d[17]), "=r"(d[18]), "=r"(d[19]), "=r"(d[20]), "=r"(d[21]), "=r"(d[22]), "=r"(d[23]),
-                               "=r"(d[24]), "=r"(d[25]), "=r"(d[26]), "=r"(d[27]), "=r"(d[28]), "=r"(d[29]), "=r"(d[30]), "=r"(d[31])
-                             : "r"(addr) : "memory");
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (P.Yt) {                                   // Eq. 7's loss against the target instead of the outputs
+                tmem_ld32(addr, d);
+                if (P.Yt) {                                   // Eq. 7's loss instead of the outputs
+                    const int code = P.teacher[pr];
+                    const bool vs_target = code < 0 || code >= 256;
+                    const int tj = code >= 0 ? (code & 255) : -1;    // co-distillation: precision tj's output is a target too
+                    uint32_t dt[32];
+                    float scale_t = 0.f;
+                    if (tj >= 0) {                                // warp-uniform
+                        tmem_ld32(tmem + ((uint32_t)(quad * 32) << 16) + tj * kBN + c0, dt);
+                        scale_t = (float)(1 << P.sh[tj]);
+                    }
                     if (m < P.M) {
                         float acc = 0.f;
-                        if (tvec) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const float tv[4] = {t4[j].x, t4[j].y, t4[j].z, t4[j].w};
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    const int cc = c0 + 4 * j + u;
-                                    const float e = al[cc] * scale * __uint_as_float(d[4 * j + u]) - az[cc] * sx - tv[u];
-                                    acc = fmaf(e, e, acc);
-                                }
+                        for (int j = 0; j < 32; ++j) {
+                            if (nb + c0 + j >= P.N) continue;
+                            const float y = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx;
+                            if (vs_target) {
+                                const float tv = tvec ? reinterpret_cast<const float*>(t4)[j] : trow[j];
+                                const float e = y - tv;
+                                acc = fmaf(e, e, acc);
                             }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nb + c0 + j < P.N) {
-                                    const float e = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx - trow[j];
-                                    acc = fmaf(e, e, acc);
-                                }
+                            if (tj >= 0) {
+                                const float e = al[c0 + j] * scale_t * __uint_as_float(dt[j]) - az[c0 + j] * sx - y;
+                                acc = fmaf(e, e, acc);
+                            }
                         }
                         lacc[pr] += acc;
                     }
@@ -460,7 +469,7 @@ static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K,
                            const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
                            const void* X, int64_t M, int64_t ldx,
                            const int* rs, int n_r, float* const* Y, int64_t ldy,
-                           const float* Yt, int64_t ldt, float* loss_part,
+                           const float* Yt, int64_t ldt, float* loss_part, const int* teacher,
                            void* workspace, size_t workspace_bytes,
                            int32_t* dev_status, void* stream) {
     using namespace matq;
@@ -546,6 +555,7 @@ static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K,
     P.alpha = alpha; P.zero = zero; P.sx = sx;
     for (int i = 0; i < kMaxR; ++i) { P.Y[i] = Y ? Y[i < n_r ? i : 0] : nullptr; P.sh[i] = c - rs[i < n_r ? i : 0]; }
     P.Yt = Yt; P.ldt = ldt; P.loss_part = loss_part;
+    for (int i = 0; i < kMaxR; ++i) P.teacher[i] = (teacher && i < n_r) ? teacher[i] : -1;
     P.M = M; P.N = N; P.K = K; P.ldy = ldy; P.n_r = n_r;
     P.dev_status = dev_status;
     // A single plane would leave every MMA at N = 128 (shared-memory bound); the CTA then takes 256 channels as two
@@ -574,7 +584,7 @@ extern "C" int matq_gemm_multi(int src_kind, const void* Wsrc, int64_t N, int64_
                                int32_t* dev_status, void* stream) {
     if (!Y) return MATQ_ERR_INVALID_ARG;
     return gemm_multi_impl(src_kind, Wsrc, N, K, c, alpha, zero, extra_precision, ovf_row_ptr, ovf_col, X, M, ldx, rs, n_r,
-                           Y, ldy, nullptr, 0, nullptr, workspace, workspace_bytes, dev_status, stream);
+                           Y, ldy, nullptr, 0, nullptr, nullptr, workspace, workspace_bytes, dev_status, stream);
 }
 
 extern "C" size_t matq_gemm_multi_loss_workspace_bytes(int src_kind, int64_t M, int64_t N, int64_t K, int n_r) {
@@ -588,7 +598,7 @@ extern "C" int matq_gemm_multi_loss(int src_kind, const void* Wsrc, int64_t N, i
                                     float* alpha, float* zero, int extra_precision,
                                     const int32_t* ovf_row_ptr, const uint16_t* ovf_col,
                                     const void* X, int64_t M, int64_t ldx,
-                                    const int* rs, int n_r, const float* lambda,
+                                    const int* rs, int n_r, const float* lambda, const int* teacher,
                                     const float* Yt, int64_t ldt, double* loss,
                                     void* workspace, size_t workspace_bytes,
                                     int32_t* dev_status, void* stream) {
@@ -596,6 +606,11 @@ extern "C" int matq_gemm_multi_loss(int src_kind, const void* Wsrc, int64_t N, i
     using namespace matq::gm;
     if (!lambda || !loss || !Yt || n_r < 1 || n_r > kMaxR || M < 0 || N < 0 || K <= 0) return MATQ_ERR_INVALID_ARG;
     if (src_kind < MATQ_SRC_BF16 || src_kind > MATQ_SRC_PACKED) return MATQ_ERR_INVALID_ARG;
+    if (teacher)
+        for (int i = 0; i < n_r; ++i) {
+            const int j = teacher[i] >= 256 ? teacher[i] - 256 : teacher[i];
+            if (teacher[i] < -1 || j >= n_r || j == i) return MATQ_ERR_INVALID_ARG;
+        }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (M == 0 || N == 0)                                        // nothing to compare: every loss is zero
         return cudaMemsetAsync(loss, 0, (size_t)(n_r + 1) * sizeof(double), s) == cudaSuccess ? MATQ_OK : MATQ_ERR_CUDA;
@@ -604,7 +619,7 @@ extern "C" int matq_gemm_multi_loss(int src_kind, const void* Wsrc, int64_t N, i
     const Layout L = layout(src_kind, M, N, K, n_r);
     float* part = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + loss_part_off(L));
     const int st = gemm_multi_impl(src_kind, Wsrc, N, K, c, alpha, zero, extra_precision, ovf_row_ptr, ovf_col, X, M, ldx,
-                                   rs, n_r, nullptr, 0, Yt, ldt, part, workspace, L.total, dev_status, stream);
+                                   rs, n_r, nullptr, 0, Yt, ldt, part, teacher, workspace, L.total, dev_status, stream);
     if (st != MATQ_OK) return st;
     LossArgs A;
     A.n_r = n_r;

@@ -114,6 +114,21 @@ def test_loss_matches_the_definition(M, N, K, rs):
         assert np.isclose(got[i], want, rtol=1e-4)
 
 
+@pytest.mark.parametrize("teacher", [(-1, 0, 0), (-1, -1, 1), (-1, 0, 256), (-1, 256, 257)])
+def test_loss_with_co_distillation_targets(teacher):
+    M, N, K = 200, 264, 256
+    W = synth.normal_bf16((N, K), 0.02, 90)
+    X = synth.normal_bf16((M, K), 1.0, 91)
+    Yt = (synth.bf16_bits_to_f32(X).astype(np.float64) @ synth.bf16_bits_to_f32(W).astype(np.float64).T).astype(np.float32)
+    lam = (1.0, 0.5, 2.0)
+    st, L_ref, total_ref, _, _ = ref.gemm_multi_loss(ref.SRC_BF16, W, K, X, Yt, lam, teacher=teacher)
+    loss, _, _ = mq.gemm_multi_loss(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), dev(Yt), lam, teacher=teacher)
+    got = host(loss)
+    assert np.allclose(got[:-1], L_ref, rtol=2e-3) and np.isclose(got[-1], total_ref, rtol=2e-3), (got, L_ref)
+    with pytest.raises(mq.MatqError):
+        mq.gemm_multi_loss(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X), dev(Yt), lam, teacher=(-1, 1, 0))   # a precision cannot teach itself
+
+
 def test_loss_is_zero_against_its_own_int8_forward_in_the_integer_case():
     rng = np.random.default_rng(9)
     N, K, M = 136, 128, 70
