@@ -212,19 +212,32 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     }
                     if (m < P.M) {
                         float acc = 0.f;
+                        if (vs_target && tvec) {                  // the common case: a whole, aligned chunk of the target
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (nb + c0 + j >= P.N) continue;
-                            const float y = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx;
-                            if (vs_target) {
-                                const float tv = tvec ? reinterpret_cast<const float*>(t4)[j] : trow[j];
-                                const float e = y - tv;
-                                acc = fmaf(e, e, acc);
+                            for (int j = 0; j < 8; ++j) {
+                                const float tv[4] = {t4[j].x, t4[j].y, t4[j].z, t4[j].w};
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int cc = c0 + 4 * j + u;
+                                    const float e = al[cc] * scale * __uint_as_float(d[4 * j + u]) - az[cc] * sx - tv[u];
+                                    acc = fmaf(e, e, acc);
+                                }
                             }
-                            if (tj >= 0) {
-                                const float e = al[c0 + j] * scale_t * __uint_as_float(dt[j]) - az[c0 + j] * sx - y;
-                                acc = fmaf(e, e, acc);
-                            }
+                        } else if (vs_target) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + c0 + j < P.N) {
+                                    const float e = al[c0 + j] * scale * __uint_as_float(d[j]) - az[c0 + j] * sx - trow[j];
+                                    acc = fmaf(e, e, acc);
+                                }
+                        }
+                        if (tj >= 0) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + c0 + j < P.N) {          // alpha z sum(x) is common to both outputs
+                                    const float e = al[c0 + j] * (scale_t * __uint_as_float(dt[j]) - scale * __uint_as_float(d[j]));
+                                    acc = fmaf(e, e, acc);
+                                }
                         }
                         lacc[pr] += acc;
                     }
