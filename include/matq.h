@@ -63,8 +63,9 @@ enum matq_gemv_flags {
     MATQ_GEMV_TCGEN05 = 3,     /* tcgen05.mma path: unpacked weights as the TMEM A operand */
     MATQ_GEMV_PATH_MASK = 0xff,
     MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
-                                  fetching weights while the previous kernel in the stream drains and
-                                  waits for it only before reading x */
+                                  fetching weights (plane, alpha, zero, overflow lists) while the previous
+                                  kernel in the stream drains and waits for it only before reading x.
+                                  Only valid when that previous kernel does not write those weights. */
 };
 
 const char *matq_status_string(int status);
@@ -78,16 +79,19 @@ int64_t matq_packed_row_bytes(int64_t K, int r);
  * (1) MinMax quantisation, Eq. 1, one (alpha, z) per output channel:
  *       alpha_n = (max_k W[n,k] - min_k W[n,k]) / (2^c - 1),  z_n = -min_k W[n,k] / alpha_n,
  *       q[n,k]  = clamp(round_half_up(W[n,k] / alpha_n + z_n), 0, 2^c - 1)
- *     evaluated in IEEE binary32, one correctly rounded operation per step in
- *     the order written (true division, no fused multiply-add).  A constant row
- *     gets alpha = 1, z = -W[n,0], codes 0.
+ *     with the result of IEEE binary32 arithmetic, one correctly rounded operation
+ *     per step in the order written (true division, separate sum): the codes are
+ *     defined bit for bit.  (The kernels may reach those bits by other instruction
+ *     sequences that reproduce every rounding.)  A constant row gets alpha = 1,
+ *     z = -W[n,0], codes 0.
  *   W      in   bf16 [N, K], row stride ldw elements (ldw >= K)
  *   q      out  uint8 [N, K] contiguous; may be NULL when only alpha / zero are wanted
  *   alpha  out  fp32 [N]
  *   zero   out  fp32 [N]
  *   A NaN / Inf weight sets dev_status = MATQ_ERR_NONFINITE; that row's outputs are unspecified.
- *   Fast path: W and q 16-byte aligned, K % 16 == 0, ldw % 8 == 0, K <= 65536.  Any other
- *   shape runs a scalar kernel.  c must be 8.
+ *   Fast paths: W 16-byte aligned, q 8-byte aligned, K % 8 == 0, ldw % 8 == 0, K <= 16384 (rows held in
+ *   registers); W and q 16-byte aligned, K % 16 == 0, ldw % 8 == 0, K <= 65536 (rows held in shared memory).
+ *   Any other shape runs a scalar kernel.  c must be 8.
  */
 int matq_quantize(const void *W, int64_t N, int64_t K, int64_t ldw, int c,
                   uint8_t *q, float *alpha, float *zero,
