@@ -3,6 +3,25 @@
 #include "gemv_cuda_core.cuh"
 #include "gemv_tensor.cuh"
 #include "gemv_tcgen05.cuh"
+#include "gemv_imma.cuh"
+
+namespace {
+
+// The integer kernel at the (m-tiles per warp, K split) the caller chose.
+template <int R>
+int launch_imma_split(int mt, int sk, const uint8_t* packed, int64_t N, int64_t K, const float* alpha, const float* zero,
+                      const int32_t* ovf_row_ptr, const uint16_t* ovf_col, const void* x, int B, int64_t ldx,
+                      float* y, int64_t ldy, bool pdl, cudaStream_t s) {
+    using namespace matq::imma;
+#define MATQ_IMMA(MT, SK, W) launch<R, MT, SK, W>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+    if (sk == 32) return MATQ_IMMA(1, 32, 32);
+    if (sk == 16) return MATQ_IMMA(1, 16, 16);
+    if (mt == 2) return sk == 8 ? MATQ_IMMA(2, 8, 8) : sk == 4 ? MATQ_IMMA(2, 4, 8) : sk == 2 ? MATQ_IMMA(2, 2, 8) : MATQ_IMMA(2, 1, 8);
+    return sk == 8 ? MATQ_IMMA(1, 8, 8) : sk == 4 ? MATQ_IMMA(1, 4, 8) : sk == 2 ? MATQ_IMMA(1, 2, 8) : MATQ_IMMA(1, 1, 8);
+#undef MATQ_IMMA
+}
+
+}  // namespace
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
     (void)N; (void)K; (void)r; (void)B;
@@ -24,7 +43,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     if (ovf_row_ptr && K > 65536) return MATQ_ERR_SHAPE;
     if ((N > 0 && !aligned16(packed)) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
     const unsigned path = flags & MATQ_GEMV_PATH_MASK;
-    if (path > MATQ_GEMV_TCGEN05 || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
+    if (path > MATQ_GEMV_TENSOR_INT8 || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
@@ -63,7 +82,19 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         if ((tiles32 * sk + 7) / 8 > 2 * sms) sk = 8;     // not even SK = 1 fits: several waves of the finest split
         while (sk > 1 && n_qc < sk) sk /= 2;
     }
-    int st;
+    int st = MATQ_ERR_SHAPE;
+    // The smallest batches go to the integer tensor path (twice the weights per MMA, one mask per four weights and
+    // no offset to remove); it declines (MATQ_ERR_SHAPE) what it does not take and the bf16 kernel below runs
+    // instead.  Measured on B200 it wins or ties at B = 1 on every decode shape (1.2-1.7x on 25-50 MB planes); at
+    // B = 2 its staging of six digit columns costs more than it saves for long rows and few channels.
+    const bool int8_auto = B == 1 || (B == 2 && K <= 4096 && N >= 8192);
+    if (((path == MATQ_GEMV_AUTO && int8_auto) || path == MATQ_GEMV_TENSOR_INT8) && B <= matq::imma::kMaxB) {
+        st = (r == 8) ? launch_imma_split<8>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+           : (r == 4) ? launch_imma_split<4>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+                      : launch_imma_split<2>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);
+        if (st == MATQ_OK) return launch_status();
+        if (st != MATQ_ERR_SHAPE) return st;
+    }
 #define MATQ_GEMV_T(RR, MT, NT, SK) launch_gemv_tensor<RR, MT, NT, SK>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
 #define MATQ_GEMV_W(RR, NT, W) launch_gemv_tensor<RR, 1, NT, W, W>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
 #define MATQ_GEMV_S(RR, MT, NT) ((sk == 8) ? MATQ_GEMV_T(RR, MT, NT, 8) : (sk == 4) ? MATQ_GEMV_T(RR, MT, NT, 4) : (sk == 2) ? MATQ_GEMV_T(RR, MT, NT, 2) : MATQ_GEMV_T(RR, MT, NT, 1))

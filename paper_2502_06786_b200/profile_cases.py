@@ -1,6 +1,8 @@
 """Small, self-contained invocations of each kernel for profilers (ncu wants short runs with few launches).
 
-    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemm
+    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemv4t|gemv2t|gemm
+
+(gemv4 / gemv2: the library's own choice at B = 1, the integer tensor kernel; a trailing t: the bf16 tensor kernel.)
 
 Every case touches a few hundred MB of distinct buffers (more than the L2 holds) and launches each kernel 16-24 times.
 """
@@ -35,8 +37,9 @@ def main(which: str) -> None:
                     mq.slice_pack(q, 4)
                 else:
                     mq.slice_pack(q, 2, extra_precision=True, ovf_capacity=N * K // 16)
-    elif which in ("gemv4", "gemv2", "gemv2b8"):
-        r = 4 if which == "gemv4" else 2
+    elif which in ("gemv4", "gemv2", "gemv2b8", "gemv4t", "gemv2t"):
+        r = 4 if which.startswith("gemv4") else 2
+        flags = mq.GEMV_TENSOR if which.endswith("t") else mq.GEMV_AUTO
         B = 8 if which.endswith("b8") else 1
         n = 24
         P = _planes(n, N, K, r)
@@ -45,7 +48,7 @@ def main(which: str) -> None:
         a = torch.ones(N, device="cuda")
         for _ in range(2):
             for i in range(n):
-                mq.gemv(P[i], K, r, a, a, X[i], y=Y[i])
+                mq.gemv(P[i], K, r, a, a, X[i], y=Y[i], flags=flags)
     elif which == "gemm":
         N2, K2, M2 = 14336, 4096, 1024      # the Mistral-7B matrix with a quarter of the tokens
         q = torch.randint(0, 256, (N2, K2), dtype=torch.uint8, device="cuda")
