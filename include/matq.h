@@ -61,9 +61,10 @@ enum matq_gemv_flags {
     MATQ_GEMV_CUDA_CORE = 1,   /* fp32 FMA path */
     MATQ_GEMV_TENSOR = 2,      /* warp-level tensor-core path (mma.sync, bf16 x bf16 -> fp32) */
     MATQ_GEMV_TCGEN05 = 3,     /* tcgen05.mma path: unpacked weights as the TMEM A operand */
-    MATQ_GEMV_TENSOR_INT8 = 4, /* warp-level integer tensor-core path (mma.sync, u8 x s8 -> s32) for B <= 4: the
-                                  fields enter as exact 8-bit integers, each activation column as two or three
-                                  base-256 digits of a block-scaled integer; larger B runs the bf16 kernel */
+    MATQ_GEMV_TENSOR_INT8 = 4, /* warp-level integer tensor-core path (mma.sync, u8 x u8 -> s32) for B = 1 and
+                                  K <= 32768: the fields enter as exact 8-bit integers, the activations as the
+                                  four bytes of a block-scaled 30-bit integer, sums are exact; anything else
+                                  runs the bf16 kernel.  MATQ_GEMV_AUTO takes this path when it applies. */
     MATQ_GEMV_PATH_MASK = 0xff,
     MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
                                   fetching weights (plane, alpha, zero, overflow lists) while the previous

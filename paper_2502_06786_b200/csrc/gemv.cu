@@ -83,12 +83,12 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         while (sk > 1 && n_qc < sk) sk /= 2;
     }
     int st = MATQ_ERR_SHAPE;
-    // The smallest batches go to the integer tensor path (twice the weights per MMA, one mask per four weights and
-    // no offset to remove); it declines (MATQ_ERR_SHAPE) what it does not take and the bf16 kernel below runs
-    // instead.  Measured on B200 it wins or ties at B = 1 on every decode shape (1.2-1.7x on 25-50 MB planes); at
-    // B = 2 its staging of six digit columns costs more than it saves for long rows and few channels.
-    const bool int8_auto = B == 1 || (B == 2 && K <= 4096 && N >= 8192);
-    if (((path == MATQ_GEMV_AUTO && int8_auto) || path == MATQ_GEMV_TENSOR_INT8) && B <= matq::imma::kMaxB) {
+    // A single activation vector goes to the integer tensor path (twice the weights per MMA, one mask per four
+    // weights, no offset to remove, exact sums); it declines (MATQ_ERR_SHAPE) what it does not take (B > 1,
+    // K > 32768) and the bf16 kernel below runs instead.  Measured on B200 it wins or ties on every decode shape
+    // (1.2-1.7x on 25-50 MB planes).
+    const bool int8_auto = B == 1;
+    if ((path == MATQ_GEMV_AUTO && int8_auto) || path == MATQ_GEMV_TENSOR_INT8) {
         st = (r == 8) ? launch_imma_split<8>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
            : (r == 4) ? launch_imma_split<4>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
                       : launch_imma_split<2>(mt, sk, packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s);

@@ -1,5 +1,5 @@
-// Decode GEMV for the smallest batches (B = 1, 2) on the integer tensor path:
-// warp-level mma.m16n8k32, u8 x s8 -> s32.
+// Decode GEMV for a single activation vector (B = 1) on the integer tensor
+// path: warp-level mma.m16n8k32, u8 x u8 -> s32.
 //
 // Why integers.  A warp-level MMA consumes one A fragment per instruction,
 // whatever the batch is, so the rate at which packed weights can be multiplied
@@ -8,22 +8,24 @@
 // with ONE mask per four weights and no shift (r = 8: nothing at all): a field
 // left where it sits in its byte reads as field * 2^s, which is still an
 // unsigned 8-bit integer, and the matching activation is divided by 2^s when it
-// is turned into an integer.  There is no offset to remove afterwards, and the
-// accumulators are 32-bit integers.
+// is turned into an integer.  The accumulators are 32-bit integers, so the
+// weights side and every sum are exact.
 //
-// The activations are bf16 and have to become 8-bit operands too.  Per batch
-// column the kernel takes e = exponent of max |x|, scales the column by the
-// power of two 2^(29 - e - s) (s = bit offset of the field the activation
-// meets, 0 <= s <= 6), rounds to an integer v with |v| < 2^30 and writes v in
-// balanced base 256: v = 2^24 t0 + 2^16 t1 + 2^8 t2 + t3, every digit in
-// [-128, 127].  Each digit is one column of the MMA's 8-wide B operand, so a
-// batch column costs four of the 8 columns and the products are summed exactly;
-// the digits are recombined in a 64-bit integer in the epilogue and scaled back
-// once.  bf16 has 8 significant bits, so every activation within 2^(-22+s) of
-// the column's largest is represented exactly and the rest to an absolute
-// 2^(-30+s) of it: a column with an outlier thousands of times its typical
-// entry still comes out at fp32 accuracy.  (Columns whose largest magnitude is
-// below 2^-97 are scaled as if it were 2^-97.)
+// The activations are bf16 and have to become 8-bit operands too.  The kernel
+// takes e = exponent of max |x|, scales x[k] by the power of two 2^(29 - e - s)
+// (s = bit offset of the field that x[k] meets, 0 <= s <= 6), rounds to an
+// integer v[k] with |v[k]| < 2^(30-s) and adds 2^(30-s): the result is a
+// non-negative 32-bit integer whose four BYTES are four columns of the MMA's
+// 8-wide B operand (byte d weighs 256^d).  A fifth column holds the constants
+// 2^(smax - s) and so returns 2^smax * (sum of the row's fields), which removes
+// the added offsets exactly:
+//   sum_k f 2^s (v + 2^(30-s)) = sum_k f 2^s v + 2^30 sum_k f.
+// The five column sums are recombined in a 64-bit integer in the epilogue and
+// scaled back once.  bf16 has 8 significant bits, so every activation within
+// 2^(-22+s) of the largest is represented exactly and the rest to an absolute
+// 2^(-30+s) of it: a vector with an outlier thousands of times its typical
+// entry still comes out at fp32 accuracy.  (A vector whose largest magnitude
+// is below 2^-97 is scaled as if it were 2^-97.)
 //
 // Fragment mapping (k slots of an MMA may be any weights as long as A and B
 // agree): thread (g = lane / 4, t = lane % 4) loads 16 bytes of rows g and g + 8
@@ -32,10 +34,11 @@
 //   r = 4: w & 0x0f0f0f0f (even fields) and w & 0xf0f0f0f0 (odd fields, times 16)
 //          are the two A registers of a row; one MMA per word.
 //   r = 2: w & (0x03030303 << 2i) holds fields i, i+4, i+8, i+12 times 4^i; two MMAs per word.
-// The activations are staged once per CTA in shared memory as 16-byte units in
-// exactly that order (the B registers of two MMAs per unit), one unit per
-// (16 weights, digit column, t), so the inner loop reads them with one
-// conflict-free 128-bit load per two MMAs.
+// The activation bytes are staged once per CTA in shared memory as 16-byte
+// units in exactly that order (the B registers of two MMAs per unit), one unit
+// per (16 weights, byte column, t), so the inner loop reads them with one
+// conflict-free 128-bit load per two MMAs; a 4 x 4 byte transpose (8 byte
+// permutes) turns four converted activations into one word of each column.
 //
 // Everything else follows the bf16 kernel: register streaming of the rows
 // three chunks ahead, the first chunks requested before the programmatic
@@ -50,9 +53,9 @@ namespace matq {
 namespace imma {
 
 constexpr int kCols = 8;                     // columns of the B operand
-constexpr int kMaxB = 2;                     // largest batch this kernel takes (four digit columns each)
-constexpr int kTerms = 4;                    // base-256 digits per activation
+constexpr int kBytes = 4;                    // byte columns of an activation (column 4 is the constant one)
 constexpr int kP = 29;                       // activations become integers below 2^(kP+1)
+constexpr int64_t kMaxK = 32768;             // 255 * 255 * K must stay below 2^31
 
 struct Params {
     const uint8_t* packed;
@@ -62,18 +65,16 @@ struct Params {
     const uint16_t* ovf_col;
     const __nv_bfloat16* x;
     float* y;
-    int64_t N, K, ldx, ldy;
+    int64_t N, K, ldy;
     int64_t row_bytes;
-    int B;            // batch columns
-    int ncp;          // digit columns staged: 4 (B = 1) or 8
     int n_qc;         // 64-byte chunks per row (the last one may be half full at r = 2)
     int qc_pass;      // chunks whose activations are staged at a time
     int pdl;
 };
 
-__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+__device__ __forceinline__ void mma_u8u8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -84,6 +85,13 @@ __host__ __device__ constexpr int unit_src(int p) {
     return R == 8 ? p : R == 4 ? (p & 8) + 2 * (p & 3) + ((p >> 2) & 1) : 4 * (p & 3) + (p >> 2);
 }
 
+// B registers of the constant column for MMA `sub` of a unit: 2^(smax - s) in every byte, s = bit offset of the
+// field that the byte's k slot holds (b0 meets the A register a0, b1 meets a2)
+template <int R>
+__device__ __forceinline__ uint32_t ones_b0(int sub) { return R == 8 ? 0x01010101u : R == 4 ? 0x10101010u : (sub ? 0x04040404u : 0x40404040u); }
+template <int R>
+__device__ __forceinline__ uint32_t ones_b1(int sub) { return R == 2 ? (sub ? 0x01010101u : 0x10101010u) : 0x01010101u; }
+
 template <int R, int MT, int SK, int WARPS, bool EP>
 __global__ void __launch_bounds__(WARPS * 32, (MT == 1 ? 32 : 16) / WARPS)
 gemv_imma(const Params P) {
@@ -93,13 +101,13 @@ gemv_imma(const Params P) {
     constexpr int kRows = kTileRows * kTiles;
     constexpr int kWpp = 128 / R;                         // weights per 16-byte piece of a row
     constexpr int kM2 = kWpp / 16;                        // staged units (pairs of MMAs) per piece
-    constexpr int sh = kCodeBits - R;
+    constexpr int sh = kCodeBits - R;                     // also the largest bit offset of a field in its byte
     constexpr int kSets = (MT >= 2) ? 1 : 2;              // independent accumulator sets per m-tile
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ uint32_t s_rmax[WARPS][kMaxB];
-    __shared__ float s_rsum[WARPS][kMaxB];
-    __shared__ float s_ep[EP ? kRows : 1][kMaxB];
+    __shared__ uint32_t s_rmax[WARPS];
+    __shared__ float s_rsum[WARPS];
+    __shared__ float s_ep[EP ? kRows : 1];
     __shared__ float s_alpha[kRows], s_zero[kRows];
     constexpr int kRowThreads = kThreads / kRows;         // = 2 SK / MT consecutive threads per row of the CTA
     constexpr int kTPR = kRowThreads > 32 ? 32 : kRowThreads;
@@ -116,16 +124,14 @@ gemv_imma(const Params P) {
         q_hi = min(q_lo + per_warp, pass_hi);
     };
     set_slice();
-    const int ncp = P.ncp;
-    constexpr int terms = kTerms;
 
-    // shared memory: staged digit units of one pass | partial tiles [warp][kTileRows][kCols]
+    // shared memory: staged byte units of one pass [chunk][unit][byte column][t] | partial tiles [warp][kTileRows][kCols]
     uint4* xs = reinterpret_cast<uint4*>(smem_raw);
-    int* part = reinterpret_cast<int*>(smem_raw + (size_t)min(P.qc_pass, P.n_qc) * kM2 * ncp * 64);
+    int* part = reinterpret_cast<int*>(smem_raw + (size_t)min(P.qc_pass, P.n_qc) * kM2 * kBytes * 64);
 
     // ---- weights of the first chunks are requested before anything that depends on the previous kernel.
     // Rows past N are clamped to the last row (never stored); a piece that would start past the end of a half-full
-    // last chunk is clamped to the row's last 16 bytes and meets activations staged as zeros.
+    // last chunk is clamped to the row's last 16 bytes and meets zeros in every column of B.
     const uint8_t* wrow[2 * MT];
 #pragma unroll
     for (int h = 0; h < 2 * MT; ++h) {
@@ -171,53 +177,35 @@ gemv_imma(const Params P) {
     float ep_x0 = 0.f;
     if (EP && ep_p < ep_hi) ep_x0 = __bfloat162float(P.x[ep_c0]);
 
-    // ---- per batch column: largest magnitude (as a bf16 bit pattern, which orders like the value) and fp32 sum
-    uint32_t cmax[kMaxB];
-    float csum[kMaxB];
+    // ---- largest magnitude (as a bf16 bit pattern, which orders like the value) and fp32 sum of the activations
+    uint32_t xmax = 0;
+    float xsum = 0.f;
     {
         const int n8 = (int)(P.K >> 3);
-#pragma unroll
-        for (int b = 0; b < kMaxB; ++b) {
-            uint32_t mx = 0;
-            float sm = 0.f;
-            if (b < P.B) {
-                const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
-                for (int i = tid; i < n8; i += kThreads) {
-                    const uint4 v = ld_x4(xr + 8 * i);
-                    mx = __vmaxu2(mx, v.x & 0x7fff7fffu); mx = __vmaxu2(mx, v.y & 0x7fff7fffu);
-                    mx = __vmaxu2(mx, v.z & 0x7fff7fffu); mx = __vmaxu2(mx, v.w & 0x7fff7fffu);
-                    sm += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) +
-                          ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
-                }
-                mx = max(mx & 0xffffu, mx >> 16);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                }
-                if (lane == 0) { s_rmax[warp][b] = mx; s_rsum[warp][b] = sm; }
-            }
-            cmax[b] = 0; csum[b] = 0.f;
+        for (int i = tid; i < n8; i += kThreads) {
+            const uint4 v = ld_x4(P.x + 8 * i);
+            xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
+            xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
+            xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
         }
+        xmax = max(xmax & 0xffffu, xmax >> 16);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+        }
+        if (lane == 0) { s_rmax[warp] = xmax; s_rsum[warp] = xsum; }
         __syncthreads();
+        xmax = lane < WARPS ? s_rmax[lane] : 0u;
+        xsum = lane < WARPS ? s_rsum[lane] : 0.f;
 #pragma unroll
-        for (int b = 0; b < kMaxB; ++b) {
-            if (b < P.B) {
-                uint32_t mx = lane < WARPS ? s_rmax[lane][b] : 0u;
-                float sm = lane < WARPS ? s_rsum[lane][b] : 0.f;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                }
-                cmax[b] = mx; csum[b] = sm;
-            }
+        for (int o = 16; o > 0; o >>= 1) {
+            xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
         }
     }
-    // biased exponent of the column's largest magnitude, kept where both 2^(P - e) and 2^(e - P) are normal floats
-    int cexp[kMaxB];
-#pragma unroll
-    for (int b = 0; b < kMaxB; ++b) cexp[b] = min(max((int)(cmax[b] >> 7), kP + 1), 254);
+    // biased exponent of the largest magnitude, kept where both 2^(P - e - s) and 2^(e - P) are normal floats
+    const int xexp = min(max((int)(xmax >> 7), kP + 1), 254);
 
     int acc[kSets][MT][4];
 #pragma unroll
@@ -228,72 +216,58 @@ gemv_imma(const Params P) {
             for (int i = 0; i < 4; ++i) acc[c][mt][i] = 0;
 
     for (;;) {
-        // ---- stage the digit units of this pass.  Item = (chunk, unit of the piece, batch column, t): 16 consecutive
-        // activations, scaled, rounded, split into digits, bytes permuted into fragment order.
+        // ---- stage the byte units of this pass.  Item = (chunk, unit of the piece, t): 16 consecutive activations,
+        // scaled, rounded, made non-negative; 4 x 4 byte transposes put byte d of four of them into one word of column d.
         {
-            const int n_items = (pass_hi - pass_lo) * kM2 * P.B * 4;
+            const int n_items = (pass_hi - pass_lo) * kM2 * 4;
+            // multiplier and offset of the activations that meet a field at bit offset R * cls of its byte
+            float mult[8 / R];
+#pragma unroll
+            for (int cls = 0; cls < 8 / R; ++cls) mult[cls] = __uint_as_float((uint32_t)(254 + kP - xexp - R * cls) << 23);
             for (int it = tid; it < n_items; it += kThreads) {
                 const int tt = it & 3;
-                const int rest = it >> 2;
-                const int b = rest % P.B;
-                const int qm = rest / P.B;                // (chunk of the pass) * kM2 + unit
+                const int qm = it >> 2;                   // (chunk of the pass) * kM2 + unit
                 const int ql = qm / kM2, m2 = qm % kM2;
                 const int k0 = ((pass_lo + ql) * 4 + tt) * kWpp + m2 * 16;
-                uint32_t digit[4][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
+                uint32_t col[kBytes][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
                 if (k0 < (int)P.K) {                      // K % 128 == 0: a unit lies inside or outside
-                    int e = cexp[0];
-#pragma unroll
-                    for (int bb = 1; bb < kMaxB; ++bb) if (b == bb) e = cexp[bb];
-                    // multiplier of the activations that meet a field at bit offset R * cls of its byte
-                    float mult[8 / R];
-#pragma unroll
-                    for (int cls = 0; cls < 8 / R; ++cls) mult[cls] = __uint_as_float((uint32_t)(254 + kP - e - R * cls) << 23);
-                    const __nv_bfloat16* xp = P.x + (int64_t)b * P.ldx + k0;
-                    const uint4 va = ld_x4(xp), vb = ld_x4(xp + 8);
+                    const uint4 va = ld_x4(P.x + k0), vb = ld_x4(P.x + k0 + 8);
                     const uint32_t raw[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-                    int v[16];
+                    uint32_t v[16];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        v[2 * i] = __float2int_rn(bf_lo(raw[i]) * mult[(2 * i) % (8 / R)]);
-                        v[2 * i + 1] = __float2int_rn(bf_hi(raw[i]) * mult[(2 * i + 1) % (8 / R)]);
+                    for (int i = 0; i < 16; ++i) {
+                        const int cls = i % (8 / R);
+                        const float xf = (i & 1) ? bf_hi(raw[i >> 1]) : bf_lo(raw[i >> 1]);
+                        v[i] = (uint32_t)(__float2int_rn(xf * mult[cls]) + (1 << (kP + 1 - R * cls)));
                     }
 #pragma unroll
-                    for (int p = 0; p < 16; ++p) {
-                        int val = v[unit_src<R>(p)];
-                        // balanced base 256, least significant digit first; digit d goes to column terms-1-d
-                        const uint32_t d0 = (uint32_t)val & 0xffu;  val = (val + 128) >> 8;
-                        const uint32_t d1 = (uint32_t)val & 0xffu;  val = (val + 128) >> 8;
-                        const uint32_t d2 = (uint32_t)val & 0xffu;  val = (val + 128) >> 8;
-                        const uint32_t d3 = (uint32_t)val & 0xffu;
-                        digit[0][p >> 2] |= d0 << (8 * (p & 3));
-                        digit[1][p >> 2] |= d1 << (8 * (p & 3));
-                        digit[2][p >> 2] |= d2 << (8 * (p & 3));
-                        digit[3][p >> 2] |= d3 << (8 * (p & 3));
+                    for (int w = 0; w < 4; ++w) {
+                        const uint32_t e0 = v[unit_src<R>(4 * w)], e1 = v[unit_src<R>(4 * w + 1)];
+                        const uint32_t e2 = v[unit_src<R>(4 * w + 2)], e3 = v[unit_src<R>(4 * w + 3)];
+                        const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e2, e3, 0x5140);
+                        const uint32_t t2 = __byte_perm(e0, e1, 0x7362), t3 = __byte_perm(e2, e3, 0x7362);
+                        col[0][w] = __byte_perm(t0, t1, 0x5410);  col[1][w] = __byte_perm(t0, t1, 0x7632);
+                        col[2][w] = __byte_perm(t2, t3, 0x5410);  col[3][w] = __byte_perm(t2, t3, 0x7632);
                     }
                 }
-                uint4* dst = xs + ((size_t)qm * ncp + b * terms) * 4 + tt;
-                dst[0] = make_uint4(digit[3][0], digit[3][1], digit[3][2], digit[3][3]);
-                dst[4] = make_uint4(digit[2][0], digit[2][1], digit[2][2], digit[2][3]);
-                dst[8] = make_uint4(digit[1][0], digit[1][1], digit[1][2], digit[1][3]);
-                dst[12] = make_uint4(digit[0][0], digit[0][1], digit[0][2], digit[0][3]);
+                uint4* dst = xs + (size_t)qm * kBytes * 4 + tt;
+#pragma unroll
+                for (int d = 0; d < kBytes; ++d) dst[4 * d] = make_uint4(col[d][0], col[d][1], col[d][2], col[d][3]);
             }
         }
         if (EP && pass_lo == 0) {                             // uniform over the CTA
-            for (int b = 0; b < P.B; ++b) {
-                const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
-                float ev = b == 0 ? ep_x0 : (ep_p < ep_hi ? __bfloat162float(xr[ep_c0]) : 0.f);
-                for (int p = ep_p + kTPR; p < ep_hi; p += 4 * kTPR) {      // lists longer than kTPR entries
-                    int col[4];
+            float ev = ep_x0;
+            for (int p = ep_p + kTPR; p < ep_hi; p += 4 * kTPR) {      // lists longer than kTPR entries
+                int col[4];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) col[u] = p + u * kTPR < ep_hi ? (int)P.ovf_col[p + u * kTPR] : -1;
+                for (int u = 0; u < 4; ++u) col[u] = p + u * kTPR < ep_hi ? (int)P.ovf_col[p + u * kTPR] : -1;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (col[u] >= 0) ev += __bfloat162float(xr[col[u]]);
-                }
-#pragma unroll
-                for (int o = kTPR / 2; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
-                if (ep_j == 0) s_ep[ep_row][b] = ev;
+                for (int u = 0; u < 4; ++u)
+                    if (col[u] >= 0) ev += __bfloat162float(P.x[col[u]]);
             }
+#pragma unroll
+            for (int o = kTPR / 2; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
+            if (ep_j == 0) s_ep[ep_row] = ev;
         }
         const bool last_pass = pass_hi >= P.n_qc;            // uniform over the CTA
         __syncthreads();
@@ -308,10 +282,12 @@ gemv_imma(const Params P) {
 #pragma unroll
                     for (int h = 0; h < 2 * MT; ++h) wv[h] = wbuf[d][h];
                     load_chunk(q + kGemvDepth, wbuf[d]);
+                    const bool piece_ok = q * 64 + t * 16 <= max_off;      // else: the clamped piece of a half-full chunk
 #pragma unroll
                     for (int m2 = 0; m2 < kM2; ++m2) {
                         uint4 xb = make_uint4(0, 0, 0, 0);
-                        if (g < ncp) xb = xs[((size_t)(q - pass_lo) * kM2 + m2) * ncp * 4 + g * 4 + t];
+                        if (g < kBytes) xb = xs[((size_t)(q - pass_lo) * kM2 + m2) * kBytes * 4 + g * 4 + t];
+                        else if (g == kBytes && piece_ok) xb = make_uint4(ones_b0<R>(0), ones_b1<R>(0), ones_b0<R>(1), ones_b1<R>(1));
 #pragma unroll
                         for (int sub = 0; sub < 2; ++sub) {
                             const uint32_t b0 = sub ? xb.z : xb.x, b1 = sub ? xb.w : xb.y;
@@ -333,7 +309,7 @@ gemv_imma(const Params P) {
                                         a1 = w_hi & (0x03030303u << (4 * sub));  a3 = w_hi & (0x0c0c0c0cu << (4 * sub));
                                     }
                                 }
-                                mma_u8s8(acc[sub % kSets][mt], a0, a1, a2, a3, b0, b1);
+                                mma_u8u8(acc[sub % kSets][mt], a0, a1, a2, a3, b0, b1);
                             }
                         }
                     }
@@ -356,7 +332,7 @@ gemv_imma(const Params P) {
             for (int i = 0; i < 4; ++i) acc[0][mt][i] += acc[1][mt][i];
     }
 
-    // ---- epilogue.  Accumulator i of thread (g, t): row g + 8*(i>>1) of the m-tile, digit column 2t + (i&1).
+    // ---- epilogue.  Accumulator i of thread (g, t): row g + 8*(i>>1) of the m-tile, column 2t + (i&1).
     {
         int* mine = part + (size_t)warp * kTileRows * kCols;
 #pragma unroll
@@ -366,27 +342,24 @@ gemv_imma(const Params P) {
         }
     }
     __syncthreads();
-    // Output o = (row of the CTA) * kMaxB + batch column: the SK partial sums of each digit column are added as
-    // integers in a fixed order, the digits recombined in 64 bits, converted once and scaled back.
-    for (int o = tid; o < kRows * kMaxB; o += kThreads) {
-        const int b = o % kMaxB, row_l = o / kMaxB;
+    // One thread per row: the SK partial sums of each column are added as integers in a fixed order, the byte columns
+    // recombined in 64 bits, the offsets removed with the constant column, one conversion, one scaling back.
+    for (int row_l = tid; row_l < kRows; row_l += kThreads) {
         const int64_t row = (int64_t)blockIdx.x * kRows + row_l;
-        if (b >= P.B || row >= P.N) continue;
-        const int* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kCols + b * terms;
-        long long tot = 0;
-        for (int d = 0; d < terms; ++d) {
-            int sd = src[d];
+        if (row >= P.N) continue;
+        const int* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kCols;
+        int sd[kBytes + 1];
 #pragma unroll
-            for (int sidx = 1; sidx < SK; ++sidx) sd += src[(size_t)sidx * kTileRows * kCols + d];
-            tot = tot * 256 + sd;
+        for (int d = 0; d <= kBytes; ++d) {
+            sd[d] = src[d];
+#pragma unroll
+            for (int sidx = 1; sidx < SK; ++sidx) sd[d] += src[(size_t)sidx * kTileRows * kCols + d];
         }
-        int e = cexp[0];
-        float sx = csum[0];
-#pragma unroll
-        for (int bb = 1; bb < kMaxB; ++bb) if (b == bb) { e = cexp[bb]; sx = csum[bb]; }
-        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(e - kP) << 23);
-        if (EP) v += s_ep[row_l][b];
-        P.y[(int64_t)b * P.ldy + row] = s_alpha[row_l] * (v * (float)(1 << sh) - s_zero[row_l] * sx);
+        // sum_k f 2^s v = sum_d 256^d D_d - 2^30 sum_k f, and column 4 holds 2^sh sum_k f
+        const long long tot = (((long long)sd[3] * 256 + sd[2]) * 256 + sd[1]) * 256 + sd[0] - ((long long)sd[4] << (kP + 1 - sh));
+        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp - kP) << 23);
+        if (EP) v += s_ep[row_l];
+        P.y[row] = s_alpha[row_l] * (v * (float)(1 << sh) - s_zero[row_l] * xsum);
     }
 }
 
@@ -398,20 +371,18 @@ inline int launch(const uint8_t* packed, int64_t N, int64_t K, const float* alph
     constexpr int kThreads = WARPS * 32;
     constexpr int kRows = 16 * MT * (WARPS / SK);
     constexpr int kM2 = (128 / R) / 16;
-    if (B < 1 || B > kMaxB) return MATQ_ERR_SHAPE;
+    (void)ldx;
+    if (B != 1 || K > kMaxK) return MATQ_ERR_SHAPE;
     Params P;
     P.packed = packed; P.alpha = alpha; P.zero = zero; P.ovf_row_ptr = ovf_row_ptr; P.ovf_col = ovf_col;
     P.x = static_cast<const __nv_bfloat16*>(x); P.y = y;
-    P.N = N; P.K = K; P.ldx = ldx; P.ldy = ldy;
+    P.N = N; P.K = K; P.ldy = ldy;
     P.row_bytes = K * R / 8;
-    if (K > 65536) return MATQ_ERR_SHAPE;                  // 255 * 128 * K must stay below 2^31 (240 * 128 * K at r = 4)
-    P.B = B;
-    P.ncp = B * kTerms;
     P.n_qc = (int)((P.row_bytes + 63) / 64);
     P.pdl = pdl ? 1 : 0;
-    // Shared memory: the staged units of one pass (64 * kM2 * ncp bytes per chunk) + the partial tiles.
+    // Shared memory: the staged units of one pass (64 * kM2 * kBytes bytes per chunk) + the partial tiles.
     const size_t part_bytes = (size_t)WARPS * 16 * MT * kCols * sizeof(int);
-    const size_t chunk_bytes = (size_t)kM2 * P.ncp * 64;
+    const size_t chunk_bytes = (size_t)kM2 * kBytes * 64;
     const int fit = (int)((150 * 1024 - part_bytes) / chunk_bytes);
     const int passes = (P.n_qc + fit - 1) / fit;
     P.qc_pass = (P.n_qc + passes - 1) / passes;
