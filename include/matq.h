@@ -160,7 +160,10 @@ int matq_slice_pack(const uint8_t *q, int64_t N, int64_t K, int c, int r, int ex
  *   y            out  fp32 [B, N], row stride ldy elements
  *   workspace         device scratch of at least matq_gemv_workspace_bytes(...) bytes (may be NULL if that is 0)
  *   flags             matq_gemv_flags
- *   fp32 accumulation; results differ from an fp64 evaluation by rounding only.
+ *   Results differ from an fp64 evaluation by rounding only.  B = 1 (and K <= 32768) sums exact integer
+ *   products of the fields with the activations scaled to 30-bit integers by a power of two taken from
+ *   max |x| (an activation below 2^-22 of the largest is rounded to an absolute 2^-24 of the largest at worst),
+ *   then applies alpha and z in fp32; other batches accumulate bf16 x bf16 products in fp32.
  */
 size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B);
 int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
