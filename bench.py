@@ -446,13 +446,15 @@ def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
     # independently, so stacking changes no result); 4 launches per layer instead of 7
     d, ff = per_layer[0][1], per_layer[4][0]
     fused_layer = [(per_layer[0][0] + per_layer[1][0] + per_layer[2][0], d), per_layer[3], (2 * ff, d), per_layer[6]]
-    out = {"workload": f"configs[2] Gemma-2-9B decoder layer shapes x {layers} layers, B = 1, one CUDA graph per precision, PDL; "
+    out = {"workload": f"configs[2] Gemma-2-9B decoder layer shapes x {layers} layers, r = 8, 4, 2 at B = 1 and r = 4, 2 at B = 4, 16, "
+                       "one CUDA graph per case, PDL; "
                        "'_fused' = q,k,v and gate,up stacked into one matrix each (4 launches per layer)"}
-    for r, fused in ((4, False), (2, False), (4, True), (2, True)):
+    for r, fused, B in ((8, False, 1), (4, False, 1), (2, False, 1), (8, True, 1), (4, True, 1), (2, True, 1),
+                        (4, False, 4), (2, False, 4), (4, False, 16), (2, False, 16)):
         shapes = [s for _ in range(layers) for s in (fused_layer if fused else per_layer)]
         planes = [torch.randint(0, 256, (n, k * r // 8), dtype=torch.uint8, device="cuda") for n, k in shapes]
-        xs = [torch.randn(1, k, device="cuda").to(torch.bfloat16) for n, k in shapes]
-        ys = [torch.empty(1, n, device="cuda") for n, k in shapes]
+        xs = [torch.randn(B, k, device="cuda").to(torch.bfloat16) for n, k in shapes]
+        ys = [torch.empty(B, n, device="cuda") for n, k in shapes]
         al = [torch.ones(n, device="cuda") for n, k in shapes]
 
         def run():
@@ -475,8 +477,8 @@ def gemv_cfg3(mq, torch, peaks, layers=6, reps=10):
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
-        nbytes = sum(bytes_gemv(n, k, r, 1) for n, k in shapes)
-        out[f"r{r}_b1" + ("_fused" if fused else "")] = {"ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
+        nbytes = sum(bytes_gemv(n, k, r, B) for n, k in shapes)
+        out[f"r{r}_b{B}" + ("_fused" if fused else "")] = {"ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1),
                            "frac_hbm": round(nbytes / ms / 1e6 / peaks["hbm_gbs"], 4), "launches": len(shapes)}
         del planes, xs, ys, al, g
         torch.cuda.empty_cache()

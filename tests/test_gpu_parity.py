@@ -329,6 +329,15 @@ def test_gemv_default_dispatch_at_benchmark_shapes(r, N, K, B, ep):
     assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
 
 
+@pytest.mark.parametrize("r", [8, 2])
+def test_gemv_default_dispatch_rows_too_long_for_integer_sums(r):
+    # K = 65536 is beyond what the integer path's 32-bit sums allow; the library's own choice must still be right.
+    y, y_ref = _gemv_case(20, 65536, 1, r, 770 + r, flags=mq.GEMV_AUTO)
+    assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
+    y, y_ref = _gemv_case(20, 65536, 1, r, 770 + r, flags=mq.GEMV_TENSOR_INT8)
+    assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
+
+
 def test_gemv_default_dispatch_on_random_shapes():
     # Ragged N, every batch size class, short and long rows, with and without overflow lists: the split heuristic has
     # many branches (SK = 1 .. 32, one or two m-tiles, 8 / 16 / 32 warps) and each must give the oracle's result.
