@@ -101,6 +101,21 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
 #define MATQ_GEMV_R(MT, NT) ((r == 8) ? MATQ_GEMV_S(8, MT, NT) : (r == 4) ? MATQ_GEMV_S(4, MT, NT) : MATQ_GEMV_S(2, MT, NT))
 #define MATQ_GEMV_RW(NT, W) ((r == 8) ? MATQ_GEMV_W(8, NT, W) : (r == 4) ? MATQ_GEMV_W(4, NT, W) : MATQ_GEMV_W(2, NT, W))
     const bool wide = mt == 2 && sk == 8 && B > 4 && B <= 8 && ((N + 31) / 32 + 1) / 2 <= sms;
+    // Batches of four or more on long rows: a cluster of 4 CTAs takes four times the rows and splits K four ways, so
+    // each CTA stages a quarter of the B activation columns (same number of CTAs, same work per warp).  Measured on
+    // B200: 3584 x 14336 at B = 8 33.5 -> 16.9 us, 3584 x 4096 at B = 16 19.4 -> 11.1 us; shapes with so few rows that
+    // a row tile has a whole CTA of 32 warps (2304 x 9216) lose with clusters (10.4 -> 14.3 us) and keep the plain kernel.
+    if (B >= 4 && n_qc >= 32 && (B >= 8 || n_qc >= 56) && (wide || sk == 16 || (mt == 2 && sk == 8))) {
+#define MATQ_GEMV_C(RR, MT, NT, SK, W) launch_gemv_tensor<RR, MT, NT, SK, W, 4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
+#define MATQ_GEMV_CR(MT, NT, SK, W) ((r == 8) ? MATQ_GEMV_C(8, MT, NT, SK, W) : (r == 4) ? MATQ_GEMV_C(4, MT, NT, SK, W) : MATQ_GEMV_C(2, MT, NT, SK, W))
+        if (wide) st = MATQ_GEMV_CR(2, 1, 2, 16);
+        else if (sk == 16) st = B <= 8 ? MATQ_GEMV_CR(1, 1, 4, 16) : MATQ_GEMV_CR(1, 2, 4, 16);
+        else st = B <= 8 ? MATQ_GEMV_CR(2, 1, 2, 8) : MATQ_GEMV_CR(2, 2, 2, 8);
+#undef MATQ_GEMV_CR
+#undef MATQ_GEMV_C
+        if (st == MATQ_OK) return launch_status();
+        if (st != MATQ_ERR_SHAPE) return st;
+    }
     if (wide) {                    // a batch: 16-warp CTAs (two row tiles) halve the staging of x' per SM (measured 4-12 %)
         st = (r == 8) ? launch_gemv_tensor<8, 2, 1, 8, 16>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)
            : (r == 4) ? launch_gemv_tensor<4, 2, 1, 8, 16>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, pdl, s)

@@ -145,7 +145,21 @@ __device__ __forceinline__ void stage_word(const __nv_bfloat16* xw, uint4* dst, 
     }
 }
 
-template <int R, int MT, int NT, int SK, int WARPS, bool EP>
+// CL > 1: a thread-block cluster of CL CTAs shares a block of rows and splits K between its CTAs, so each CTA stages
+// only 1/CL of the activations (the staging of B columns per CTA is what a batch costs); the per-CTA partial results
+// (offset already removed) are summed by the cluster's first CTA through distributed shared memory.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(const float* local, uint32_t rank) {
+    uint32_t la = (uint32_t)__cvta_generic_to_shared(local), ra;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+template <int R, int MT, int NT, int SK, int WARPS, bool EP, int CL = 1>
 __global__ void __launch_bounds__(WARPS * 32, (MT == 1 ? 32 : 16) / WARPS)   // MT = 1: 64 registers, a full SM of warps
 gemv_tensor(const GemvTensorParams P) {
     constexpr int kGemvThreads = WARPS * 32, kGemvWarps = WARPS;
@@ -162,17 +176,22 @@ gemv_tensor(const GemvTensorParams P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ float s_sumx[kMaxB], s_sumxp[kMaxB], s_grp[2][kGemvThreads / 4];
     __shared__ float s_ep[EP ? kRows : 1][kMaxB];         // extra-precision correction per row and batch column
-    __shared__ float s_alpha[SK > 1 ? kRows : 1], s_zero[SK > 1 ? kRows : 1];
+    __shared__ float s_alpha[(SK > 1 || CL > 1) ? kRows : 1], s_zero[(SK > 1 || CL > 1) ? kRows : 1];
     constexpr int kRowThreads = kGemvThreads / kRows;     // = 2 SK / MT consecutive threads per row of the CTA
     constexpr int kTPR = kRowThreads > 32 ? 32 : kRowThreads;   // of which this many walk the row's overflow list
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int tile = warp / SK, ks = warp % SK;
-    const int64_t row0 = (int64_t)blockIdx.x * kRows + (int64_t)tile * kTileRows;
+    uint32_t crank = 0;                                   // this CTA's place in its cluster = its share of K
+    if (CL > 1) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+    const int64_t rblock = CL > 1 ? (int64_t)(blockIdx.x / CL) : (int64_t)blockIdx.x;   // block of kRows rows
+    const int64_t row0 = rblock * kRows + (int64_t)tile * kTileRows;
+    const int c_per = (P.n_qc + CL - 1) / CL;
+    const int c_lo = min((int)crank * c_per, P.n_qc), c_hi = min(c_lo + c_per, P.n_qc);   // this CTA's chunks
     // K is walked in passes of qc_pass chunks (one pass unless the staged activations would not fit in shared memory);
     // inside a pass the SK warps of a row tile take consecutive slices of its chunks.
-    int pass_lo = 0, pass_hi = min(P.qc_pass, P.n_qc);
+    int pass_lo = c_lo, pass_hi = min(c_lo + P.qc_pass, c_hi);
     int q_lo, q_hi;
     auto set_slice = [&]() {
         const int per_warp = (pass_hi - pass_lo + SK - 1) / SK;
@@ -185,6 +204,7 @@ gemv_tensor(const GemvTensorParams P) {
     // shared memory: x' fragments for all of K | partial tiles [warp][kTileRows][kMaxB] (SK > 1 only)
     uint4* xs = reinterpret_cast<uint4*>(smem_raw);
     float* part = reinterpret_cast<float*>(smem_raw + (size_t)min(P.qc_pass, P.n_qc) * 4 * kPG * bpad * 64);
+    float* red = part + (size_t)kGemvWarps * kTileRows * kMaxB;     // CL > 1: [kRows][kMaxB] partial results + [kMaxB] sums of x
 
     // ---- weights of the first chunks are requested before anything that depends on the previous kernel
     // Rows past N are clamped to the last row (their results are never stored) and a lane whose piece would start
@@ -213,7 +233,7 @@ gemv_tensor(const GemvTensorParams P) {
     // scale and zero point: with SK = 1 a thread finishes rows g and g+8 of every m-tile from its accumulators and
     // keeps them in registers; with SK > 1 the CTA's rows are parked in shared memory for the shared epilogue.
     float a_pre[2 * MT], z_pre[2 * MT];
-    if (SK == 1) {
+    if (SK == 1 && CL == 1) {
 #pragma unroll
         for (int h = 0; h < 2 * MT; ++h) {
             const int64_t row = row0 + (h >> 1) * 16 + (h & 1) * 8 + g;
@@ -222,7 +242,7 @@ gemv_tensor(const GemvTensorParams P) {
         }
     } else {
         for (int rl = tid; rl < kRows; rl += kGemvThreads) {
-            const int64_t row = (int64_t)blockIdx.x * kRows + rl;
+            const int64_t row = rblock * kRows + rl;
             s_alpha[rl] = row < P.N ? P.alpha[row] : 0.f;
             s_zero[rl] = row < P.N ? P.zero[row] : 0.f;
         }
@@ -234,8 +254,8 @@ gemv_tensor(const GemvTensorParams P) {
     // barrier that precedes the epilogue.
     const int ep_row = tid / kRowThreads, ep_j = tid % kRowThreads;
     int ep_p = 0, ep_hi = 0, ep_c0 = 0;
-    if (EP && ep_j < kTPR) {
-        const int64_t row = (int64_t)blockIdx.x * kRows + ep_row;
+    if (EP && ep_j < kTPR && crank == 0) {
+        const int64_t row = rblock * kRows + ep_row;
         if (row < P.N) {
             ep_p = P.ovf_row_ptr[row] + ep_j;
             ep_hi = P.ovf_row_ptr[row + 1];
@@ -289,7 +309,7 @@ gemv_tensor(const GemvTensorParams P) {
                 }
             }
         }
-        if (EP && pass_lo == 0) {                             // uniform over the CTA
+        if (EP && pass_lo == 0 && crank == 0) {               // uniform over the CTA
             for (int b = 0; b < P.B; ++b) {
                 const __nv_bfloat16* xr = P.x + (int64_t)b * P.ldx;
                 float ev = b == 0 ? ep_x0 : (ep_p < ep_hi ? __bfloat162float(xr[ep_c0]) : 0.f);
@@ -306,7 +326,7 @@ gemv_tensor(const GemvTensorParams P) {
                 if (ep_j == 0) s_ep[ep_row][b] = ev;
             }
         }
-        const bool last_pass = pass_hi >= P.n_qc;            // uniform over the CTA
+        const bool last_pass = pass_hi >= c_hi;              // uniform over the CTA
         if (last_pass) {
             sx += __shfl_xor_sync(0xffffffffu, sx, 1);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 1);
             sx += __shfl_xor_sync(0xffffffffu, sx, 2);  sxp += __shfl_xor_sync(0xffffffffu, sxp, 2);
@@ -373,7 +393,7 @@ gemv_tensor(const GemvTensorParams P) {
         if (last_pass) break;
         // ---- next pass: request its first chunks, then wait until every warp is done with the staged activations
         pass_lo = pass_hi;
-        pass_hi = min(pass_lo + P.qc_pass, P.n_qc);
+        pass_hi = min(pass_lo + P.qc_pass, c_hi);
         set_slice();
 #pragma unroll
         for (int d = 0; d < kGemvDepth; ++d) load_chunk(q_lo + d, wbuf[d]);
@@ -389,7 +409,7 @@ gemv_tensor(const GemvTensorParams P) {
     }
 
     // ---- epilogue.  Accumulator i of thread (g, t): row g + 8*(i>>1) of the m-tile, batch column 2t + (i&1).
-    if (SK > 1) {
+    if (SK > 1 || CL > 1) {
         float* mine = part + (size_t)warp * kTileRows * kMaxB;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -400,12 +420,42 @@ gemv_tensor(const GemvTensorParams P) {
                     mine[(mt * 16 + g + (i >> 1) * 8) * kMaxB + nt * 8 + 2 * t + (i & 1)] = acc[0][mt][nt][i];
     }
     __syncthreads();                                      // publishes s_sumx / s_sumxp and the partial tiles
+    if (CL > 1) {
+        // this CTA's share of every output, offset removed (everything is linear in the K range), and of the sums of x
+        for (int o = tid; o < kRows * kMaxB; o += kGemvThreads) {
+            const int b = o % kMaxB, row_l = o / kMaxB;
+            const float* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kMaxB + b;
+            float v = src[0];
+#pragma unroll
+            for (int sidx = 1; sidx < SK; ++sidx) v += src[(size_t)sidx * kTileRows * kMaxB];
+            red[o] = v - 128.0f * s_sumxp[b];
+        }
+        if (tid < kMaxB) red[kRows * kMaxB + tid] = s_sumx[tid];
+        cluster_sync_all();
+        if (crank == 0) {
+            for (int o = tid; o < kRows * kMaxB; o += kGemvThreads) {
+                const int b = o % kMaxB, row_l = o / kMaxB;
+                const int64_t row = rblock * kRows + row_l;
+                if (b >= P.B || row >= P.N) continue;
+                float v = red[o], sxa = red[kRows * kMaxB + b];
+#pragma unroll
+                for (uint32_t c = 1; c < (uint32_t)CL; ++c) {
+                    v += ld_cluster_f32(red + o, c);
+                    sxa += ld_cluster_f32(red + kRows * kMaxB + b, c);
+                }
+                if (EP) v += s_ep[row_l][b];
+                P.y[(int64_t)b * P.ldy + row] = s_alpha[row_l] * (v * (float)(1 << sh) - s_zero[row_l] * sxa);
+            }
+        }
+        cluster_sync_all();                               // the other CTAs' shared memory stays alive until it was read
+        return;
+    }
     if (SK > 1) {
         // Every thread finishes outputs: output o = (row of the CTA) * kMaxB + batch column sums its SK partials in
         // a fixed order and is scaled with the row's alpha / zero (parked in shared memory at the start).
         for (int o = tid; o < kRows * kMaxB; o += kGemvThreads) {
             const int b = o % kMaxB, row_l = o / kMaxB;
-            const int64_t row = (int64_t)blockIdx.x * kRows + row_l;
+            const int64_t row = rblock * kRows + row_l;
             if (b >= P.B || row >= P.N) continue;
             const float* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kMaxB + b;
             float v = src[0];
@@ -434,7 +484,7 @@ gemv_tensor(const GemvTensorParams P) {
 }
 
 // Host side: geometry and launch.
-template <int R, int MT, int NT, int SK, int WARPS = 8>
+template <int R, int MT, int NT, int SK, int WARPS = 8, int CL = 1>
 inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const float* alpha, const float* zero,
                               const int32_t* ovf_row_ptr, const uint16_t* ovf_col, const void* x, int B, int64_t ldx,
                               float* y, int64_t ldy, bool pdl, cudaStream_t s) {
@@ -455,26 +505,37 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     P.bpad_log2 = P.bpad == 1 ? 0 : P.bpad == 2 ? 1 : P.bpad == 4 ? 2 : P.bpad == 8 ? 3 : 4;
     // Shared memory: the staged activations of one pass (64 * 4 * kPG * bpad bytes per chunk) + the split-K partials.
     // Passes are as long as ~150 KB allow (one pass for all decode shapes up to K = 9216 at B = 8).
-    const size_t part_bytes = SK > 1 ? (size_t)kGemvWarps * 16 * MT * kMaxB * sizeof(float) : 0;
+    const size_t part_bytes = (SK > 1 || CL > 1 ? (size_t)kGemvWarps * 16 * MT * kMaxB * sizeof(float) : 0) +
+                              (CL > 1 ? (size_t)(kRows + 1) * kMaxB * sizeof(float) : 0);
     const size_t chunk_bytes = (size_t)4 * kPG * P.bpad * 64;
     const int fit = (int)((150 * 1024 - part_bytes) / chunk_bytes);
-    const int passes = (P.n_qc + fit - 1) / fit;
-    P.qc_pass = (P.n_qc + passes - 1) / passes;
+    const int c_per = (P.n_qc + CL - 1) / CL;             // chunks of one CTA of a cluster
+    const int passes = (c_per + fit - 1) / fit;
+    P.qc_pass = (c_per + passes - 1) / passes;
     const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
-    auto kern = ovf_row_ptr ? gemv_tensor<R, MT, NT, SK, WARPS, true> : gemv_tensor<R, MT, NT, SK, WARPS, false>;
+    auto kern = ovf_row_ptr ? gemv_tensor<R, MT, NT, SK, WARPS, true, CL> : gemv_tensor<R, MT, NT, SK, WARPS, false, CL>;
     if (smem > 16 * 1024 &&   // the 48 KB default counts static shared memory too
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows), 1, 1);
+    cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows) * CL, 1, 1);
     cfg.blockDim = dim3(kGemvThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (CL > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = CL; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = pdl ? 1 : 0;
+    cfg.numAttrs = na;
     if (cudaLaunchKernelEx(&cfg, kern, P) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
     return MATQ_OK;
 }

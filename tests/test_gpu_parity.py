@@ -329,6 +329,17 @@ def test_gemv_default_dispatch_at_benchmark_shapes(r, N, K, B, ep):
     assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
 
 
+@pytest.mark.parametrize("r", [8, 4, 2])
+@pytest.mark.parametrize("N,K,B,ep", [(5001, 4096, 8, True), (5000, 4096, 16, False), (4801, 8192, 4, False),
+                                      (3000, 4096, 12, True), (3584, 14336, 8, True), (2500, 8192, 5, False)])
+def test_gemv_batches_on_long_rows_split_k_over_a_cluster(r, N, K, B, ep):
+    # B >= 4 on long rows: clusters of 4 CTAs split K and the first CTA sums the partial results through distributed
+    # shared memory.  Every cluster variant (one / two m-tiles, 8 / 16 warps, one / two n-tiles), ragged N, overflow lists.
+    ep = ep and r < 8
+    y, y_ref = _gemv_case(N, K, B, r, 880 + r + B, ep=ep, flags=mq.GEMV_AUTO | mq.GEMV_PDL)
+    assert np.abs(y - y_ref).max() <= TOL_TENSOR * rms(y_ref)
+
+
 @pytest.mark.parametrize("r", [8, 2])
 def test_gemv_default_dispatch_rows_too_long_for_integer_sums(r):
     # K = 65536 is beyond what the integer path's 32-bit sums allow; the library's own choice must still be right.
