@@ -342,21 +342,25 @@ gemv_imma(const Params P) {
         }
     }
     __syncthreads();
-    // One thread per row: the SK partial sums of each column are added as integers in a fixed order, the byte columns
-    // recombined in 64 bits, the offsets removed with the constant column, one conversion, one scaling back.
-    for (int row_l = tid; row_l < kRows; row_l += kThreads) {
+    // One thread per (row, column): the SK partial sums of a column are added as integers in a fixed order; the
+    // five columns of a row sit in neighbouring lanes and are recombined in 64 bits by the first of them, the
+    // offsets removed with the constant column, one conversion, one scaling back.  kRows * kCols is a multiple of
+    // 32, so whole warps take part in the shuffles.
+    for (int o = tid; o < kRows * kCols; o += kThreads) {
+        const int col = o % kCols, row_l = o / kCols;
         const int64_t row = (int64_t)blockIdx.x * kRows + row_l;
-        if (row >= P.N) continue;
-        const int* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kCols;
-        int sd[kBytes + 1];
+        const int* src = part + ((size_t)(row_l / kTileRows) * SK * kTileRows + row_l % kTileRows) * kCols + col;
+        int sd = 0;
+        if (col <= kBytes) {
+            sd = src[0];
 #pragma unroll
-        for (int d = 0; d <= kBytes; ++d) {
-            sd[d] = src[d];
-#pragma unroll
-            for (int sidx = 1; sidx < SK; ++sidx) sd[d] += src[(size_t)sidx * kTileRows * kCols + d];
+            for (int sidx = 1; sidx < SK; ++sidx) sd += src[(size_t)sidx * kTileRows * kCols];
         }
+        const int s1 = __shfl_down_sync(0xffffffffu, sd, 1, kCols), s2 = __shfl_down_sync(0xffffffffu, sd, 2, kCols);
+        const int s3 = __shfl_down_sync(0xffffffffu, sd, 3, kCols), s4 = __shfl_down_sync(0xffffffffu, sd, 4, kCols);
+        if (col != 0 || row >= P.N) continue;
         // sum_k f 2^s v = sum_d 256^d D_d - 2^30 sum_k f, and column 4 holds 2^sh sum_k f
-        const long long tot = (((long long)sd[3] * 256 + sd[2]) * 256 + sd[1]) * 256 + sd[0] - ((long long)sd[4] << (kP + 1 - sh));
+        const long long tot = (((long long)s3 * 256 + s2) * 256 + s1) * 256 + sd - ((long long)s4 << (kP + 1 - sh));
         float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp - kP) << 23);
         if (EP) v += s_ep[row_l];
         P.y[row] = s_alpha[row_l] * (v * (float)(1 << sh) - s_zero[row_l] * xsum);
