@@ -53,6 +53,23 @@ __device__ __forceinline__ uint32_t pack4(uint32_t k) {
     return (t | (t >> 12)) & 0xffu;
 }
 
+// r = 2 in one step: four codes -> the packed byte of their four clamped 2-bit fields and the 4-bit mask of the codes
+// whose Eq. 8 value is one bucket higher.  With u = q >> 6 (bits 7, 6) and the rounding bit t = bit 5, Eq. 6 is
+// min(u + t, 3), i.e. bit 1 = u1 | (u0 & t), bit 0 = (u0 ^ t) | (u1 & u0 & t), overflow = u1 & u0 & t: three
+// bitwise functions of the word and its shifts by one and two, evaluated for all four bytes at once (only bits 7
+// and 6 of each byte are kept, so what the shifts carry across byte borders never matters).  The multiplications
+// gather bits 7, 6 of the four bytes into the top byte, and bit 7 of the four bytes into the top nibble; the partial
+// products land on distinct bits, so nothing carries.
+__device__ __forceinline__ void slice_pack4_r2(uint32_t w, uint32_t& byte, uint32_t& ovmask) {
+    const uint32_t l1 = w << 1, l2 = w << 2, r1 = w >> 1;
+    const uint32_t ovw = w & l1 & l2;
+    const uint32_t k1 = w | (l1 & l2);
+    const uint32_t k0 = (w ^ l1) | (r1 & w & l1);
+    const uint32_t kk = (k1 & 0x80808080u) | (k0 & 0x40404040u);
+    byte = (kk * 0x00041041u) >> 24;
+    ovmask = ((ovw & 0x80808080u) * 0x00204081u) >> 28;
+}
+
 // bits 0, 8, 16, 24 -> bits 0..3
 __device__ __forceinline__ uint32_t gather_byte_lsbs(uint32_t ov) { return ((ov * 0x01020408u) >> 24) & 0xfu; }
 
@@ -67,6 +84,16 @@ slice_pack_vec(const uint4* __restrict__ q, int64_t nchunks, int chunks_per_row,
     const int64_t stride = (int64_t)gridDim.x * kSliceThreads;
     for (int64_t i = (int64_t)blockIdx.x * kSliceThreads + threadIdx.x; i < nchunks; i += stride) {
         const uint4 v = ld_stream_u4(q + i);
+        if (PACK_R == 2 && !sliced) {
+            uint32_t b0, b1, b2, b3, m0, m1, m2, m3;
+            slice_pack4_r2(v.x, b0, m0); slice_pack4_r2(v.y, b1, m1); slice_pack4_r2(v.z, b2, m2); slice_pack4_r2(v.w, b3, m3);
+            reinterpret_cast<uint32_t*>(packed)[i] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+            if (row_count) {
+                const int cnt = __popc(m0 | (m1 << 4) | (m2 << 8) | (m3 << 12));
+                if (cnt) atomicAdd(row_count + (i / chunks_per_row), cnt);
+            }
+            continue;
+        }
         const Sliced s0 = slice4(v.x, r), s1 = slice4(v.y, r), s2 = slice4(v.z, r), s3 = slice4(v.w, r);
         if (PACK_R == 8) {
             reinterpret_cast<uint4*>(packed)[i] = make_uint4(s0.k, s1.k, s2.k, s3.k);
@@ -346,6 +373,16 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
                     for (int u = 0; u < kEpBatch; ++u) {
                         const int c = c0 + u * 32 + lane;
                         if (c >= cpr) continue;
+                        if (PACK_R == 2 && !sliced) {
+                            uint32_t b0, b1, b2, b3, m0, m1, m2, m3;
+                            slice_pack4_r2(v[u].x, b0, m0); slice_pack4_r2(v[u].y, b1, m1);
+                            slice_pack4_r2(v[u].z, b2, m2); slice_pack4_r2(v[u].w, b3, m3);
+                            reinterpret_cast<uint32_t*>(packed)[c_row + c] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                            const uint32_t m = m0 | (m1 << 4) | (m2 << 8) | (m3 << 12);
+                            mrow[c] = (uint16_t)m;
+                            cnt += __popc(m);
+                            continue;
+                        }
                         const Sliced s0 = slice4(v[u].x, r), s1 = slice4(v[u].y, r), s2 = slice4(v[u].z, r), s3 = slice4(v[u].w, r);
                         if (PACK_R == 4) {
                             reinterpret_cast<uint2*>(packed)[c_row + c] =
