@@ -65,6 +65,9 @@ enum matq_gemv_flags {
                                   K <= 32768: the fields enter as exact 8-bit integers, the activations as the
                                   four bytes of a block-scaled 30-bit integer, sums are exact; anything else
                                   runs the bf16 kernel.  MATQ_GEMV_AUTO takes this path when it applies. */
+    MATQ_GEMV_STREAM = 5,      /* persistent integer tensor-core kernel (B = 1, K <= 32768): one CTA per SM, the plane
+                                  streamed by bulk copies into a ring in shared memory; the kernel behind
+                                  matq_gemv_grouped, here with a list of one */
     MATQ_GEMV_PATH_MASK = 0xff,
     MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
                                   fetching weights (plane, alpha, zero, overflow lists) while the previous
@@ -172,6 +175,42 @@ int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
               const void *x, int B, int64_t ldx, float *y, int64_t ldy,
               void *workspace, size_t workspace_bytes, unsigned flags,
               int32_t *dev_status, void *stream);
+
+/*
+ * (3b) Several decode GEMVs (B = 1) in ONE launch.  A decoder layer multiplies the same activation vector with
+ *      several weight matrices (the query, key and value projections; the gate and up projections of the FFN,
+ *      Sections 1 and 5.3), a Mix'n'Match model (Section 3.2.1, Appendix B) gives every layer its own r, and each
+ *      plane is only a few megabytes, i.e. a few microseconds of HBM time: a launch per plane is bound by launch
+ *      latency, not by the weight traffic that Section 1 names as the cost of decoding.  This call takes a list of
+ *      independent problems, each exactly a matq_gemv with B = 1,
+ *        y_i[n] = sum_k x_i[k] * alpha_i[n] * (S_i[n,k] - z_i[n])        (+ Eq. 8's extra bucket where a list is given),
+ *      and runs them with one persistent kernel whose CTAs share the list's bytes evenly, whatever the shapes.
+ *      Problems may share x or not, may differ in N, K and r, and must not depend on one another (no y_i may be
+ *      an x_j of the same call).  Results are those of matq_gemv's integer path (exact integer sums, reproducible,
+ *      independent of how the list is split over CTAs).
+ *   problems   in   HOST array of n_problems descriptors; the pointers inside are DEVICE pointers:
+ *                     packed uint8 [N, K*r/8] 16-byte aligned, alpha / zero fp32 [N], ovf_row_ptr / ovf_col both NULL
+ *                     or both given, x bf16 [K] 16-byte aligned, y fp32 [N].  r in {8, 4, 2}, K % 128 == 0, K <= 32768.
+ *                     A problem with N == 0 is skipped.  The array is read during the call only.
+ *   n_problems      any number >= 0; up to 128 problems share a launch, longer lists take several
+ *   flags           0 or MATQ_GEMV_PDL (meaning as for matq_gemv: no plane, alpha, zero or list of the call is
+ *                   written by the previous kernel of the stream)
+ *   A wait inside the kernel that does not end within about two seconds sets dev_status = MATQ_ERR_TIMEOUT; the
+ *   outputs are then unspecified and the kernel still returns.
+ */
+typedef struct matq_gemv_problem {
+    const uint8_t *packed;
+    int64_t N, K;
+    int r;
+    const float *alpha;
+    const float *zero;
+    const int32_t *ovf_row_ptr;
+    const uint16_t *ovf_col;
+    const void *x;
+    float *y;
+} matq_gemv_problem;
+int matq_gemv_grouped(const matq_gemv_problem *problems, int n_problems, int c, unsigned flags,
+                      int32_t *dev_status, void *stream);
 
 /*
  * (4) Multi-precision dense forward of MatQuant co-training (Eq. 7): for every

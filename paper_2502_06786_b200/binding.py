@@ -19,14 +19,21 @@ _LIB_PATH = os.path.join(_HERE, "libmatq.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_SHAPE, ERR_ALIGNMENT = 0, 1, 2, 3, 4
 ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_CAPACITY, ERR_TIMEOUT = 5, 6, 8, 9, 10
 SRC_BF16, SRC_CODES8, SRC_PACKED = 0, 1, 2
-GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_TENSOR_INT8, GEMV_PDL = 0, 1, 2, 3, 4, 0x100
+GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_TENSOR_INT8, GEMV_STREAM, GEMV_PDL = 0, 1, 2, 3, 4, 5, 0x100
 TEACHER_AND_TARGET = 256    # matq_gemm_multi_loss: teacher[i] = TEACHER_AND_TARGET + j
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
-           "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv",
+           "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
            "matq_gemm_multi_loss_workspace_bytes", "matq_gemm_multi_loss",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
+
+
+class GemvProblem(C.Structure):
+    """matq_gemv_problem."""
+    _fields_ = [("packed", C.c_void_p), ("N", C.c_int64), ("K", C.c_int64), ("r", C.c_int),
+                ("alpha", C.c_void_p), ("zero", C.c_void_p), ("ovf_row_ptr", C.c_void_p), ("ovf_col", C.c_void_p),
+                ("x", C.c_void_p), ("y", C.c_void_p)]
 
 
 class MatqError(RuntimeError):
@@ -57,6 +64,8 @@ def _load():
     lib.matq_gemv_workspace_bytes.argtypes = [i64, i64, i32, i32]
     lib.matq_gemv.restype = i32
     lib.matq_gemv.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, i32, i64, vp, i64, vp, sz, u32, vp, vp]
+    lib.matq_gemv_grouped.restype = i32
+    lib.matq_gemv_grouped.argtypes = [C.POINTER(GemvProblem), i32, i32, u32, vp, vp]
     lib.matq_gemm_multi_workspace_bytes.restype = sz
     lib.matq_gemm_multi_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
     lib.matq_gemm_multi.restype = i32
@@ -207,6 +216,35 @@ def gemv(packed, K, r, alpha, zero, x, y=None, ovf_row_ptr=None, ovf_col=None, w
                         _ptr(dev_status), _stream())
     _check(st, "matq_gemv")
     return y
+
+
+def gemv_group(problems):
+    """Descriptor array for gemv_grouped from dicts / tuples (packed, K, r, alpha, zero, x, y[, ovf_row_ptr, ovf_col]).
+    Build it once and reuse it: it holds raw pointers, the caller keeps the tensors alive."""
+    arr = (GemvProblem * len(problems))()
+    for d, pr in zip(arr, problems):
+        if isinstance(pr, dict):
+            pr = (pr["packed"], pr["K"], pr["r"], pr["alpha"], pr["zero"], pr["x"], pr["y"], pr.get("ovf_row_ptr"), pr.get("ovf_col"))
+        packed, K, r, alpha, zero, x, y = pr[:7]
+        rp, col = (pr[7], pr[8]) if len(pr) > 7 else (None, None)
+        _dev(packed, torch.uint8, "packed", 2); _dev(x, torch.bfloat16, "x"); _dev(y, torch.float32, "y")
+        _dev(alpha, torch.float32, "alpha"); _dev(zero, torch.float32, "zero")
+        if not packed.is_contiguous() or not x.is_contiguous() or not y.is_contiguous() or x.numel() != K or y.numel() != packed.shape[0]:
+            raise ValueError("packed, x [K] and y [N] must be contiguous and match the shape")
+        d.packed, d.N, d.K, d.r = packed.data_ptr(), packed.shape[0], K, r
+        d.alpha, d.zero, d.x, d.y = alpha.data_ptr(), zero.data_ptr(), x.data_ptr(), y.data_ptr()
+        d.ovf_row_ptr = None if rp is None else rp.data_ptr()
+        d.ovf_col = None if col is None else col.data_ptr()
+    return arr
+
+
+def gemv_grouped(group, flags=0, dev_status=None, c=8, raise_on_error=True):
+    """matq_gemv_grouped on a descriptor array from gemv_group (or a list accepted by it)."""
+    if not isinstance(group, C.Array):
+        group = gemv_group(group)
+    st = _lib.matq_gemv_grouped(group, len(group), c, int(flags), _ptr(dev_status), _stream())
+    _check(st, "matq_gemv_grouped", raise_on_error)
+    return st
 
 
 def gemm_multi_workspace_bytes(src_kind, M, N, K, n_r) -> int:

@@ -4,6 +4,7 @@
 #include "gemv_tensor.cuh"
 #include "gemv_tcgen05.cuh"
 #include "gemv_imma.cuh"
+#include "gemv_stream.cuh"
 
 namespace {
 
@@ -21,7 +22,27 @@ int launch_imma_split(int mt, int sk, const uint8_t* packed, int64_t N, int64_t 
 #undef MATQ_IMMA
 }
 
+constexpr long long kStreamWaitCycles = 4000000000ll;         // limit of its waits: about two seconds of SM clock
+
 }  // namespace
+
+extern "C" int matq_gemv_grouped(const matq_gemv_problem* problems, int n_problems, int c, unsigned flags,
+                                 int32_t* dev_status, void* stream) {
+    using namespace matq;
+    if (n_problems < 0 || (n_problems > 0 && !problems)) return MATQ_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)MATQ_GEMV_PDL) return MATQ_ERR_INVALID_ARG;
+    if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
+    static_assert(sizeof(gstream::HostProblem) == sizeof(matq_gemv_problem), "descriptor layouts must agree");
+    for (int i = 0; i < n_problems; ++i) {
+        const matq_gemv_problem& q = problems[i];
+        if (q.N < 0 || q.K <= 0 || !q.x || (q.N > 0 && (!q.packed || !q.alpha || !q.zero || !q.y))) return MATQ_ERR_INVALID_ARG;
+        if ((q.ovf_row_ptr == nullptr) != (q.ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
+        if (!(q.r == 8 || q.r == 4 || q.r == 2)) return MATQ_ERR_UNSUPPORTED;
+        if (q.K % 128 != 0 || q.K > imma::kMaxK || q.N >= (1ll << 31) - 16) return MATQ_ERR_SHAPE;
+        if ((q.N > 0 && !aligned16(q.packed)) || !aligned16(q.x)) return MATQ_ERR_ALIGNMENT;
+    }
+    return gstream::launch(reinterpret_cast<const gstream::HostProblem*>(problems), n_problems, (flags & MATQ_GEMV_PDL) != 0, kStreamWaitCycles, dev_status, static_cast<cudaStream_t>(stream));
+}
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
     (void)N; (void)K; (void)r; (void)B;
@@ -43,7 +64,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     if (ovf_row_ptr && K > 65536) return MATQ_ERR_SHAPE;
     if ((N > 0 && !aligned16(packed)) || !aligned16(x)) return MATQ_ERR_ALIGNMENT;
     const unsigned path = flags & MATQ_GEMV_PATH_MASK;
-    if (path > MATQ_GEMV_TENSOR_INT8 || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
+    if (path > MATQ_GEMV_STREAM || (flags & ~(MATQ_GEMV_PATH_MASK | MATQ_GEMV_PDL))) return MATQ_ERR_INVALID_ARG;
     if (N == 0) return MATQ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
@@ -59,6 +80,11 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else if (r == 4) st5 = t5::launch<4>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         else st5 = t5::launch<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         if (st5 != MATQ_ERR_SHAPE) return st5;     // a K too long for one cluster's shared memory falls through
+    }
+    if (path == MATQ_GEMV_STREAM) {
+        if (B != 1 || !gstream::eligible(N, K, r)) return MATQ_ERR_SHAPE;
+        const gstream::HostProblem hp = {packed, N, K, r, alpha, zero, ovf_row_ptr, ovf_col, x, y};
+        return gstream::launch(&hp, 1, pdl, kStreamWaitCycles, dev_status, s);
     }
     // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at ONE wave of CTAs
     // (a second, partly filled wave costs up to 40 %; measured on B200 for 4-26 MB planes):

@@ -1,0 +1,885 @@
+// Decode GEMV for single activation vectors (B = 1) as ONE persistent kernel
+// over a list of problems: the planes are streamed by the copy engine into a
+// ring in shared memory, the multiplies are the integer warp MMAs of
+// gemv_imma.cuh.
+//
+// Why.  A packed plane of a decoder layer is 2-50 MB, i.e. 0.4-8 us of HBM
+// time, and a kernel per plane spends about 2 us per launch on a chain that no
+// amount of tuning removes (dependency wait, activations, multiply, K-split
+// sum, store, drain).  Here
+//   * one CTA per SM stays resident for the whole list; each CTA owns a
+//     contiguous share of the list's (16-row tile x 64-byte chunk) items, cut
+//     at tile boundaries, so SMs are balanced to within one tile whatever the
+//     shapes are, and a CTA prepares the activations only of the one to three
+//     problems its share touches;
+//   * one producer warp feeds a ring of 18.5 KB stages with ONE copy per stage
+//     (completion counted on an mbarrier).  A stage is one UNIT: rows of up to
+//     1184 bytes are staged whole, 1 to 4 consecutive 16-row tiles being one
+//     contiguous run of the plane (cp.async.bulk); longer rows are cut into K
+//     panels of at most 1088 bytes and a unit is the 16 x panel box of a tensor
+//     map over the plane (cp.async.bulk.tensor.2d; rows and columns past the
+//     end arrive as zeros).  One copy per unit matters: the copy engine takes
+//     about 55 ns per request whatever its size, so a copy per row segment
+//     cannot reach the HBM rate.  150 KB and more per SM are in flight
+//     independently of what the multiplying warps do, and with programmatic
+//     dependent launch the ring is filled while the previous kernel of the
+//     stream is still running;
+//   * every unit is multiplied by ONE consumer warp (unit s of a CTA's share of
+//     a problem goes to warp s mod W, and the number of stages is a multiple of
+//     W, so a stage always serves the same warp and a warp never has to ask
+//     whether an older use of its stage has completed): A fragments come from the stage with
+//     128-bit loads, B fragments from the staged activation bytes exactly as in
+//     gemv_imma, into eight independent accumulator sets.  Warps never wait for
+//     one another while a problem is being multiplied:
+//       - when the share has at least W tiles, the units are ordered so that a
+//         warp receives all panels of "its" tiles; it keeps the sums in
+//         registers and finishes the 16 outputs alone (three shuffles per row);
+//       - when it has fewer tiles than warps and rows of several panels, the
+//         panels of a tile are spread over the warps; each adds its partial
+//         sums to a small accumulator in shared memory with integer atomics and
+//         the warp that arrives last finishes the tile.
+//     Integer sums do not depend on their order, so the result is reproducible
+//     and does not depend on how the list was cut or which warp came last.
+// The arithmetic (fields masked in place as exact 8-bit operands, activations
+// as the four bytes of a block-scaled integer, a constant column that removes
+// the offsets) is that of gemv_imma.cuh and is described there; the masks are
+// nested here (see stage_activations), which saves a quarter to a half of them.
+//
+// Extra precision (Errata, Eq. 8): a listed column's field is one bucket higher
+// than the stored, clamped one, so its activation is added once more in fp32;
+// the warp that finishes a tile walks the lists of its 16 rows.
+//
+// Every wait is bounded (a limit in clock cycles, about two seconds): a wait
+// that gives up sets a flag in shared memory and MATQ_ERR_TIMEOUT in
+// dev_status; from then on every wait returns at once, the control flow of all
+// warps (trip counts, named barriers) stays the same, nothing more is stored,
+// and the producer waits, bounded, for the copies it still has in flight before
+// the CTA returns.
+#pragma once
+#include <algorithm>
+#include <atomic>
+
+#include "common.cuh"
+#include "gemv_imma.cuh"
+#include "gemv_tcgen05.cuh"
+#include "gemv_tensor.cuh"
+
+namespace matq {
+namespace gstream {
+
+constexpr int kMaxSlots = 24;
+constexpr int kUnitBytes = 16 * 1184;        // largest unit
+constexpr int kMaxTpu = 4;                   // tiles per unit at most
+constexpr int kMaxW = 11;                    // consumer warps (with the producer: 12 warps, 168 registers a thread)
+constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
+constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
+constexpr int kSmallList = 8;
+constexpr int kLargeList = 128;
+constexpr int kSmemLimit = 227 * 1024;
+constexpr int kSets = 8;                     // independent accumulator sets of a warp
+constexpr unsigned kWaitHintNs = 2000;       // longest suspension of one probe of a stage by a multiplying warp
+constexpr unsigned kProducerNapNs = 100;     // pause of the producer warp when it has nothing to issue
+
+struct Problem {
+    const uint8_t* packed;
+    const float* alpha;
+    const float* zero;
+    const int32_t* ovf_row_ptr;
+    const uint16_t* ovf_col;
+    const __nv_bfloat16* x;
+    float* y;
+    int N, K;
+    int r;
+    int pad_;
+    long long item0;          // (tile x chunk) items of the problems before this one
+};
+
+template <int NP>
+struct Params {
+    CUtensorMap tm[NP];       // over each plane as [N][row_bytes / 8] 64-bit words, box 16 x panel (only read for long rows)
+    Problem p[NP];
+    long long items;          // total items
+    long long wait_cycles;    // limit of a wait, in SM clock cycles
+    int32_t* dev_status;
+    int n;                    // problems
+    int slots;                // ring stages in use
+    int slot_bytes;
+    int xs_bytes;             // staged activation bytes (largest problem)
+    int W;                    // consumer warps
+    int pdl;
+};
+
+// Shape of a problem's units.  Rows of up to 1184 bytes are staged whole: `tpu` (1 to 4) consecutive tiles are one
+// contiguous run of the plane, rows `row_bytes` apart in shared memory.  Longer rows are cut into `n_panels` panels
+// of `panel_qc` 64-byte chunks (an odd number, so that rows are an odd multiple of 64 bytes apart and the 128-bit
+// loads of a quarter warp fall into different banks; the last panel may be shorter), one tile per unit.
+struct Geo {
+    int row_bytes, n_qc, tiles, n_panels, panel_qc, stride, contig, tpu;
+};
+__host__ __device__ inline Geo geometry(int N, int K, int r) {
+    Geo g;
+    g.row_bytes = K / 8 * r;
+    g.n_qc = (g.row_bytes + 63) / 64;
+    g.tiles = (N + 15) / 16;
+    if (16 * g.row_bytes <= kUnitBytes) {
+        g.contig = 1;
+        g.tpu = kUnitBytes / (16 * g.row_bytes);
+        if (g.tpu > kMaxTpu) g.tpu = kMaxTpu;
+        g.n_panels = 1;
+        g.panel_qc = g.n_qc;
+        g.stride = g.row_bytes;
+        return g;
+    }
+    g.contig = 0;
+    g.tpu = 1;
+    const int max_qc = (kUnitBytes / 16) / 64 - 1;      // 17
+    g.n_panels = (g.n_qc + max_qc - 1) / max_qc;
+    g.panel_qc = (g.n_qc + g.n_panels - 1) / g.n_panels;
+    g.panel_qc |= 1;
+    g.n_panels = (g.n_qc + g.panel_qc - 1) / g.panel_qc;
+    g.stride = g.panel_qc * 64;
+    return g;
+}
+
+// How a CTA's share of a problem (T tiles, i.e. ceil(T / tpu) groups of tiles) is laid out as a sequence of units.
+// Unit s goes to warp s mod W; the sequence is padded with empty units to a multiple of W.
+//   at least W groups, or single-panel rows: rounds of W groups; within a round panel-major, so warp w meets
+//     (group g W + w, panel 0), (same group, panel 1), ...;
+//   fewer tiles than warps and several panels: tile-major, the panels of a tile are spread over the warps.
+struct Plan {
+    int split, n_units;
+};
+__host__ __device__ inline Plan plan_of(const Geo& g, int T, int W) {
+    Plan pl;
+    const int Tu = (T + g.tpu - 1) / g.tpu;
+    pl.split = (Tu < W && g.n_panels > 1) ? 1 : 0;
+    pl.n_units = pl.split ? (T * g.n_panels + W - 1) / W * W : (Tu + W - 1) / W * g.n_panels * W;
+    return pl;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// one probe of a phase; the hardware may suspend the thread for up to `hint_ns` before it answers
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
+// one probe of a phase that never suspends
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// one contiguous run of global memory into this CTA's shared memory; completion is counted in bytes on `bar`
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// the 16-row box of a tensor map that starts at (64-bit word x, row y) into this CTA's shared memory
+__device__ __forceinline__ void tensor_g2s(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// Bounded wait for phase `parity` of an mbarrier.  Returns false (and raises the abort flag) when it gives up; returns
+// false at once when another wait of this CTA already gave up.  The limit is in SM clock cycles (reading the clock
+// costs a few cycles; the nanosecond timer costs about a microsecond).
+__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles) {
+    if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+    if (*abort_flag) return false;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
+    }
+}
+
+// The next problem (from index p on) of which this CTA owns tiles, and which: [t_lo, t_hi).
+template <int NP>
+__device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, long long hi, int& p, int& t_lo, int& t_hi) {
+    while (p < P.n) {
+        const long long i0 = P.p[p].item0;
+        if (i0 >= hi) return false;
+        const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r);
+        const long long a = lo > i0 ? (lo - i0 + g.n_qc - 1) / g.n_qc : 0;
+        const long long b = (hi - i0 + g.n_qc - 1) / g.n_qc;
+        ++p;
+        t_lo = (int)(a < g.tiles ? a : g.tiles);
+        t_hi = (int)(b < g.tiles ? b : g.tiles);
+        if (t_lo < t_hi) return true;
+    }
+    return false;
+}
+
+// 128-bit shared-memory load that only the lanes with `on` execute; the others keep what `v` held.
+__device__ __forceinline__ void lds128_if(uint4& v, uint32_t addr, int on) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %5, 0;\n @p ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n}"
+                 : "+r"(v.x), "+r"(v.y), "+r"(v.z), "+r"(v.w) : "r"(addr), "r"(on));
+}
+
+// One (tile, chunk) item: 16 rows x 64 bytes of plane from the stage, times the staged activation bytes.  B source:
+// the lanes of byte column g < 4 (`col_lane`) load their column of the chunk's staged units from shared memory
+// (`x_sa`: shared address of the first unit, the next one 256 bytes further); the lanes g = 4 hold the constant
+// column in `xb` and keep it (the load is predicated off for them, which also halves the shared-memory wavefronts of
+// the B loads); what the lanes g > 4 hold is irrelevant, columns 5-7 of the product are never read.
+// The 2 * kM2 MMAs go to accumulator sets SET0, SET0 + 1, ...
+template <int R, int SET0>
+__device__ __forceinline__ void multiply_item(const unsigned char* wl_p, const unsigned char* wh_p, uint32_t x_sa, int col_lane,
+                                              uint4 (&xb)[(128 / R) / 16], int (&acc)[kSets][4]) {
+    constexpr int kM2 = (128 / R) / 16;
+    const uint4 wl = *reinterpret_cast<const uint4*>(wl_p);
+    const uint4 wh = *reinterpret_cast<const uint4*>(wh_p);
+#pragma unroll
+    for (int m2 = 0; m2 < kM2; ++m2) lds128_if(xb[m2], x_sa + m2 * 256, col_lane);
+#pragma unroll
+    for (int m2 = 0; m2 < kM2; ++m2) {
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+            const uint32_t b0 = sub ? xb[m2].z : xb[m2].x, b1 = sub ? xb[m2].w : xb[m2].y;
+            uint32_t a0, a1, a2, a3;
+            if (R == 8) {
+                a0 = sub ? wl.z : wl.x;  a2 = sub ? wl.w : wl.y;
+                a1 = sub ? wh.z : wh.x;  a3 = sub ? wh.w : wh.y;
+            } else {
+                const int j = R == 4 ? 2 * m2 + sub : m2;
+                const uint32_t w_lo = j == 0 ? wl.x : j == 1 ? wl.y : j == 2 ? wl.z : wl.w;
+                const uint32_t w_hi = j == 0 ? wh.x : j == 1 ? wh.y : j == 2 ? wh.z : wh.w;
+                // nested masks: operand i keeps fields 0 .. i of its byte (the last one is the byte as it stands)
+                if (R == 4) {
+                    a0 = w_lo & 0x0f0f0f0fu;  a2 = w_lo;
+                    a1 = w_hi & 0x0f0f0f0fu;  a3 = w_hi;
+                } else if (sub == 0) {
+                    a0 = w_lo & 0x03030303u;  a2 = w_lo & 0x0f0f0f0fu;
+                    a1 = w_hi & 0x03030303u;  a3 = w_hi & 0x0f0f0f0fu;
+                } else {
+                    a0 = w_lo & 0x3f3f3f3fu;  a2 = w_lo;
+                    a1 = w_hi & 0x3f3f3f3fu;  a3 = w_hi;
+                }
+            }
+            imma::mma_u8u8(acc[SET0 + 2 * m2 + sub], a0, a1, a2, a3, b0, b1);
+        }
+    }
+}
+
+// All chunks of one unit's tile panel.  `wl_p` / `wh_p`: this lane's 16 bytes of rows g and g + 8 in the first chunk;
+// `x_sa`: shared address of its B source for that chunk, `xq_bytes` per chunk further for the next; `cz`: the
+// constant column (lanes g = 4).  Four chunks (two at r = 2) are taken per round: their loads are issued together,
+// and the eight accumulator sets are used in turn, so that neither the shared-memory latency nor the MMA latency
+// sits between two MMAs of a warp.
+template <int R>
+__device__ __forceinline__ void multiply_unit(const unsigned char* wl_p, const unsigned char* wh_p, uint32_t x_sa, int xq_bytes, int col_lane,
+                                              const uint4& cz, int n_chunks, int (&acc)[kSets][4]) {
+    constexpr int kM2 = (128 / R) / 16;
+    constexpr int kU = R == 2 ? 2 : 4;                    // chunks per round
+    uint4 xb[kU][kM2];
+#pragma unroll
+    for (int i = 0; i < kU; ++i)
+#pragma unroll
+        for (int m2 = 0; m2 < kM2; ++m2) xb[i][m2] = cz;
+#define MATQ_ITEM(I) multiply_item<R, ((I) * 2 * kM2) % kSets>(wl_p + (c + (I)) * 64, wh_p + (c + (I)) * 64, x_sa + (c + (I)) * xq_bytes, col_lane, xb[I], acc)
+    int c = 0;
+#pragma unroll 1
+    for (; c + kU <= n_chunks; c += kU) {
+        MATQ_ITEM(0);
+        MATQ_ITEM(1);
+        if (kU >= 4) { MATQ_ITEM(2); MATQ_ITEM(3); }
+    }
+#pragma unroll 1
+    for (; c < n_chunks; ++c) MATQ_ITEM(0);
+#undef MATQ_ITEM
+}
+
+// Activation bytes of one problem in B-fragment order (all chunks of a row).  The byte layout is that of
+// gemv_imma.cuh; the values differ in one respect that saves a quarter (r = 2) or half (r = 4) of the mask
+// instructions of the multiply.  With V_i = round(x_i 2^(P - e - R i)) for the activation that meets field i of a
+// byte, gemv_imma pairs V_i with the operand f_i 2^(R i) (one mask per field).  Here operand i is the byte masked
+// to its fields 0 .. i, A_i = sum_{j <= i} f_j 2^(R j) (the last one needs no mask at all), paired with
+// Y_i = V_i - V_{i+1} (Y of the last field = V):  sum_i A_i Y_i = sum_j f_j 2^(R j) sum_{i >= j} Y_i = sum_j f_j 2^(R j) V_j,
+// the same exact integer.  |Y_i| < 1.25 * 2^(P + 1 - R i), so the offset that makes it a non-negative 32-bit
+// integer is 2^(P + 2 - R i); the constant column (2^(smax - R i) per byte) returns sum_i A_i 2^(smax - R i), which
+// removes sum_i A_i 2^(P + 2 - R i) exactly.
+template <int R>
+__device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K, int n_qc, int xexp, uint4* xs, int ctid, int nthr) {
+    constexpr int kWpp = 128 / R;
+    constexpr int kM2 = kWpp / 16;
+    constexpr int kF = 8 / R;                                  // fields per byte
+    float mult[kF];
+#pragma unroll
+    for (int cls = 0; cls < kF; ++cls) mult[cls] = __uint_as_float((uint32_t)(254 + imma::kP - xexp - R * cls) << 23);
+    const int n_items = n_qc * kM2 * 4;
+    for (int it = ctid; it < n_items; it += nthr) {
+        const int tt = it & 3;
+        const int qm = it >> 2;
+        const int ql = qm / kM2, m2 = qm % kM2;
+        const int k0 = (ql * 4 + tt) * kWpp + m2 * 16;
+        uint32_t col[imma::kBytes][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
+        if (k0 < K) {
+            const uint4 va = ld_x4(x + k0), vb = ld_x4(x + k0 + 8);
+            const uint32_t raw[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+            int V[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float xf = (i & 1) ? bf_hi(raw[i >> 1]) : bf_lo(raw[i >> 1]);
+                V[i] = __float2int_rn(xf * mult[i % kF]);
+            }
+            uint32_t v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const int cls = i % kF;                          // 16 consecutive activations start at a byte boundary
+                const int y = cls == kF - 1 ? V[i] : V[i] - V[i + 1 < 16 ? i + 1 : i];
+                v[i] = (uint32_t)y + (1u << (imma::kP + 2 - R * cls));
+            }
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const uint32_t e0 = v[imma::unit_src<R>(4 * w)], e1 = v[imma::unit_src<R>(4 * w + 1)];
+                const uint32_t e2 = v[imma::unit_src<R>(4 * w + 2)], e3 = v[imma::unit_src<R>(4 * w + 3)];
+                const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e2, e3, 0x5140);
+                const uint32_t t2 = __byte_perm(e0, e1, 0x7362), t3 = __byte_perm(e2, e3, 0x7362);
+                col[0][w] = __byte_perm(t0, t1, 0x5410);  col[1][w] = __byte_perm(t0, t1, 0x7632);
+                col[2][w] = __byte_perm(t2, t3, 0x5410);  col[3][w] = __byte_perm(t2, t3, 0x7632);
+            }
+        }
+        uint4* dst = xs + (size_t)qm * imma::kBytes * 4 + tt;
+#pragma unroll
+        for (int d = 0; d < imma::kBytes; ++d) dst[4 * d] = make_uint4(col[d][0], col[d][1], col[d][2], col[d][3]);
+    }
+}
+
+// What a consumer warp knows about the problem it is multiplying.
+struct Ctx {
+    const Problem* pr;
+    Geo G;
+    float xsum;
+    int xexp;
+    int sh;
+};
+
+// Finishes one tile.  Accumulator a_i of thread (g, t) holds row g + 8 (i >> 1), column 2t + (i & 1); the five
+// columns of a row are recombined in 64 bits by the lanes t = 0 and scaled back once.  `scales`: alpha of row
+// (lane) in lanes 0-15, zero of row (lane - 16) in lanes 16-31.  Called by whole warps.
+__device__ __noinline__ void finish_tile(const Ctx& c, long long row0, int a0, int a1, int a2, int a3, float scales, int lane, bool store) {
+    const int g = lane >> 2, t = lane & 3;
+    const Problem& pr = *c.pr;
+    // extra precision (Eq. 8): sum of the activations at the listed columns of each of the 16 rows
+    float ep_lo = 0.f, ep_hi = 0.f;
+    if (pr.ovf_row_ptr) {
+        for (int rl = 0; rl < 16; ++rl) {
+            const long long row = row0 + rl;
+            float ev = 0.f;
+            if (row < pr.N) {
+                const int e0 = pr.ovf_row_ptr[row], e1 = pr.ovf_row_ptr[row + 1];
+                for (int e = e0 + lane; e < e1; e += 32) ev += __bfloat162float(pr.x[pr.ovf_col[e]]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
+            if (rl == g) ep_lo = ev;
+            if (rl == g + 8) ep_hi = ev;
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {                               // rows g and g + 8
+        const int d0 = h ? a2 : a0, d1 = h ? a3 : a1;
+        const int d2 = __shfl_down_sync(0xffffffffu, d0, 1), d3 = __shfl_down_sync(0xffffffffu, d1, 1);
+        const int d4 = __shfl_down_sync(0xffffffffu, d0, 2);
+        const float al = __shfl_sync(0xffffffffu, scales, g + 8 * h), ze = __shfl_sync(0xffffffffu, scales, 16 + g + 8 * h);
+        const long long row = row0 + g + 8 * h;
+        if (t != 0 || row >= pr.N || !store) continue;
+        // sum_i A_i Y_i = sum_d 256^d D_d - sum_i A_i 2^(P + 2 - R i), and column 4 holds sum_i A_i 2^(sh - R i)
+        const long long tot = (((long long)d3 * 256 + d2) * 256 + d1) * 256 + d0 - ((long long)d4 << (imma::kP + 2 - c.sh));
+        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(c.xexp - imma::kP) << 23);
+        v += h ? ep_hi : ep_lo;
+        pr.y[row] = al * (v * (float)(1 << c.sh) - ze * c.xsum);
+    }
+}
+
+template <int NP>
+__global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
+gemv_stream(const __grid_constant__ Params<NP> P) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t s_full[kMaxSlots], s_empty[kMaxSlots];
+    __shared__ int s_tile[kTileSlots][16][imma::kCols];       // sums of tiles whose panels are spread over warps
+    __shared__ int s_tile_cnt[kTileSlots];
+    __shared__ uint32_t s_rmax[kMaxW];
+    __shared__ float s_rsum[kMaxW];
+    __shared__ int s_abort;
+
+    const int W = P.W;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nthr = W * 32;                                  // consumer threads
+    uint4* xs = reinterpret_cast<uint4*>(smem_raw);
+    unsigned char* ring = smem_raw + P.xs_bytes;
+    volatile int* abort_flag = &s_abort;
+
+    if (tid == 0) {
+        s_abort = 0;
+        for (int s = 0; s < P.slots; ++s) {
+            mbar_init(smem_u32(&s_full[s]), 1);
+            mbar_init(smem_u32(&s_empty[s]), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < kTileSlots * 16 * imma::kCols; i += blockDim.x) (&s_tile[0][0][0])[i] = 0;
+    if (tid < kTileSlots) s_tile_cnt[tid] = 0;
+    __syncthreads();
+    if (P.pdl) asm volatile("griddepcontrol.launch_dependents;");
+
+    // this CTA's share of the list: items [lo, hi), cut at tile boundaries (a tile belongs to the CTA its first item falls to)
+    const long long lo = P.items * blockIdx.x / gridDim.x, hi = P.items * (blockIdx.x + 1) / gridDim.x;
+    int p_first = 0;
+    {
+        int a = 0, b = P.n - 1;                               // last problem that starts at or before lo
+        while (a < b) {
+            const int m = (a + b + 1) >> 1;
+            if (P.p[m].item0 <= lo) a = m; else b = m - 1;
+        }
+        p_first = a;
+    }
+
+    if (warp == W) {
+        // ------------------------------------------------------------------ producer warp: lane l < W feeds warp l's stages
+        int it0 = 0;                                          // units of the segments before this one (a multiple of W)
+        bool waited = !P.pdl;
+        int p = p_first, t_lo, t_hi;
+        bool ok = true;
+        int last_it = -1;                                     // latest unit this lane issued a copy for
+        while (ok && next_segment(P, lo, hi, p, t_lo, t_hi)) {
+            const Problem& pr = P.p[p - 1];
+            const Geo G = geometry(pr.N, pr.K, pr.r);
+            const int T = t_hi - t_lo;
+            const Plan pl = plan_of(G, T, W);
+            // Lane l feeds warp l: its units are l, l + W, ...; (tile, panel) and (stage, phase) move by fixed steps.  The
+            // lanes advance independently: each probes ITS stage (without suspending) and issues its next copy as soon as
+            // its warp has released the stage, so a slow consumer warp never holds back the copies of the others.
+            const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
+            int tj = pl.split ? lane / G.n_panels : lane * G.tpu;
+            int pn = pl.split ? lane % G.n_panels : 0;
+            int slot = (it0 + lane) % P.slots;
+            int use = (it0 + lane) / P.slots;                      // how often the stage has been used before
+            int s = lane < W ? lane : pl.n_units;                  // this lane's next unit
+            long long t_wait = 0;
+            int spins = 0;
+            while (__any_sync(0xffffffffu, s < pl.n_units)) {
+                if (!waited && __any_sync(0xffffffffu, s < pl.n_units && use > 0)) {
+                    // The consumers only start after the previous kernel of the stream has finished; wait for it here
+                    // (a wait the stream itself bounds), so that the bounded waits below measure this CTA only.
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    waited = true;
+                }
+                bool progressed = false;
+                if (s < pl.n_units && (use == 0 || mbar_test_wait(smem_u32(&s_empty[slot]), (uint32_t)((use - 1) & 1)))) {
+                    const uint32_t bar = smem_u32(&s_full[slot]);
+                    const uint32_t dst = smem_u32(ring + (size_t)slot * P.slot_bytes);
+                    if (tj >= T) {
+                        mbar_arrive(bar);                           // padding: an empty unit
+                    } else if (G.contig) {
+                        // the unit is one run of the plane; rows past the end of the matrix are not fetched
+                        const long long row0 = (long long)(t_lo + tj) * 16;
+                        const long long rows = min((long long)min(G.tpu, T - tj) * 16, pr.N - row0);
+                        const uint32_t bytes = (uint32_t)rows * (uint32_t)G.row_bytes;
+                        mbar_arrive_expect_tx(bar, bytes);
+                        bulk_g2s(dst, pr.packed + row0 * G.row_bytes, bytes, bar);
+                        last_it = it0 + s;
+                    } else {
+                        mbar_arrive_expect_tx(bar, (uint32_t)(16 * G.stride));     // the whole box, zeros included
+                        tensor_g2s(dst, &P.tm[p - 1], pn * G.panel_qc * 8, (t_lo + tj) * 16, bar);
+                        last_it = it0 + s;
+                    }
+                    if (pl.split) {
+                        tj += step_t; pn += step_p;
+                        if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
+                    } else if (++pn == G.n_panels) { pn = 0; tj += W * G.tpu; }
+                    slot += W;
+                    if (slot >= P.slots) { slot -= P.slots; ++use; }
+                    s += W;
+                    progressed = true;
+                }
+                // bounded: no lane made progress for the wait limit
+                if (__any_sync(0xffffffffu, progressed)) { spins = 0; t_wait = 0; }
+                else {
+                    __nanosleep(kProducerNapNs);                      // every stage is full: leave the issue slots to the multiplying warps
+                    if (++spins >= 64) {
+                        spins = 0;
+                        const long long now = clock64();
+                        if (t_wait == 0) t_wait = now;
+                        const bool give_up = *abort_flag || now - t_wait > P.wait_cycles;
+                        if (__any_sync(0xffffffffu, give_up)) { *abort_flag = 1; ok = false; break; }
+                    }
+                }
+            }
+            it0 += pl.n_units;
+        }
+        if (!ok && lane < W) {
+            // gave up: copies already issued still write into this CTA's shared memory; wait for them (bounded).  A lane's
+            // stages are its own, so the phase of a stage's latest use stays complete once its copy has landed.
+            const long long t0 = clock64();
+            for (int it = last_it; it >= 0 && it > last_it - P.slots; it -= W) {
+                const uint32_t bar = smem_u32(&s_full[it % P.slots]);
+                while (!mbar_try_wait(bar, (uint32_t)((it / P.slots) & 1), 1000) && clock64() - t0 < P.wait_cycles) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumer warps
+        const int g = lane >> 2, t = lane & 3;
+        const int ctid = tid;                                  // warps 0 .. W-1
+        int it0 = 0;                                           // units of the segments before this one (a multiple of W)
+        int split_tiles = 0;                                   // split-mode tiles of earlier segments (a tile's slot = its count mod kTileSlots)
+        int p = p_first, t_lo, t_hi;
+        bool first = true;
+        Ctx c;
+        while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
+            const Problem& pr = P.p[p - 1];
+            c.pr = &pr;
+            c.G = geometry(pr.N, pr.K, pr.r);
+            const Geo& G = c.G;
+            const int R = pr.r;
+            c.sh = kCodeBits - R;
+            const int T = t_hi - t_lo;
+            const Plan pl = plan_of(G, T, W);
+            if (first && P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+            first = false;
+
+            // ---- largest magnitude and fp32 sum of the activations, then their bytes in fragment order.
+            // The first barrier also separates the previous problem's multiplies from the restaging.
+            uint32_t xmax = 0;
+            float xsum = 0.f;
+            for (int i = ctid; i < (pr.K >> 3); i += nthr) {
+                const uint4 v = ld_x4(pr.x + 8 * i);
+                xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
+                xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
+                xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
+            }
+            xmax = max(xmax & 0xffffu, xmax >> 16);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+            }
+            if (lane == 0) { s_rmax[warp] = xmax; s_rsum[warp] = xsum; }
+            asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+            xmax = lane < W ? s_rmax[lane] : 0u;
+            xsum = lane < W ? s_rsum[lane] : 0.f;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+                xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+            }
+            c.xsum = xsum;
+            c.xexp = min(max((int)(xmax >> 7), imma::kP + 1), 254);
+            if (R == 8) stage_activations<8>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
+            else if (R == 4) stage_activations<4>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
+            else stage_activations<2>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
+            asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+
+            const int kM2 = (128 / R) / 16;
+            // this lane's B source: chunk q of byte column g starts at xs[q * kM2 * 16 + g * 4 + t]; the lanes g = 4 hold
+            // the constant column (2^(smax - s) per byte, see gemv_imma.cuh) in registers
+            const int col_lane = g < imma::kBytes ? 1 : 0;
+            const uint32_t x_sa0 = smem_u32(xs) + (uint32_t)((g & 3) * 4 + t) * 16u;
+            const int xq_bytes = kM2 * 256;
+            uint4 cz = make_uint4(0, 0, 0, 0);
+            if (g == imma::kBytes) {
+                if (R == 8) cz = make_uint4(imma::ones_b0<8>(0), imma::ones_b1<8>(0), imma::ones_b0<8>(1), imma::ones_b1<8>(1));
+                else if (R == 4) cz = make_uint4(imma::ones_b0<4>(0), imma::ones_b1<4>(0), imma::ones_b0<4>(1), imma::ones_b1<4>(1));
+                else cz = make_uint4(imma::ones_b0<2>(0), imma::ones_b1<2>(0), imma::ones_b0<2>(1), imma::ones_b1<2>(1));
+            }
+            const bool half_tail = (G.row_bytes & 63) != 0;          // r = 2, K % 256 == 128: the last chunk is half full
+
+            // panel `pn` of the tile whose rows start at `tile_rows` in a stage
+            auto multiply = [&](const unsigned char* tile_rows, int pn, int (&acc)[kSets][4]) {
+                const int q0 = pn * G.panel_qc, q1 = min(q0 + G.panel_qc, G.n_qc);
+                const unsigned char* base = tile_rows + t * 16;
+                const unsigned char* wl_p = base + (size_t)g * G.stride;
+                const unsigned char* wh_p = base + (size_t)(g + 8) * G.stride;
+                const uint32_t x_sa = x_sa0 + (uint32_t)(q0 * xq_bytes);
+                int n_chunks = q1 - q0;
+                const bool tail = half_tail && q1 == G.n_qc;
+                if (tail) --n_chunks;
+                if (R == 8) multiply_unit<8>(wl_p, wh_p, x_sa, xq_bytes, col_lane, cz, n_chunks, acc);
+                else if (R == 4) multiply_unit<4>(wl_p, wh_p, x_sa, xq_bytes, col_lane, cz, n_chunks, acc);
+                else multiply_unit<2>(wl_p, wh_p, x_sa, xq_bytes, col_lane, cz, n_chunks, acc);
+                if (tail) {
+                    // the pieces t >= 2 of the half-full chunk lie past the end of the row: their activation bytes
+                    // were staged as zeros, and the constant column must be zero for them too
+                    uint4 xt[4];
+#pragma unroll
+                    for (int m2 = 0; m2 < 4; ++m2) xt[m2] = t < 2 ? cz : make_uint4(0, 0, 0, 0);
+                    multiply_item<2, 0>(wl_p + n_chunks * 64, wh_p + n_chunks * 64, x_sa + (uint32_t)(n_chunks * xq_bytes), col_lane, xt, acc);
+                }
+            };
+            auto zero_acc = [&](int (&acc)[kSets][4]) {
+#pragma unroll
+                for (int c2 = 0; c2 < kSets; ++c2)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[c2][i] = 0;
+            };
+            auto fold = [&](int (&acc)[kSets][4]) {
+#pragma unroll
+                for (int c2 = 1; c2 < kSets; ++c2)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[0][i] += acc[c2][i];
+            };
+            // alpha (lanes 0-15) and zero (lanes 16-31) of the 16 rows of a tile
+            auto load_scales = [&](long long row0) -> float {
+                const long long row = row0 + (lane & 15);
+                if (row >= pr.N) return 0.f;
+                return lane < 16 ? pr.alpha[row] : pr.zero[row];
+            };
+
+            // ---- this warp's units, in order.  One call site for the multiply and one for the finish keep the loop small
+            // enough for the instruction cache (warps are at different places of it most of the time).
+            int acc[kSets][4];
+            const int contributors = min(G.n_panels, W);              // split mode: warps that hold a part of a tile
+            int cur = -1;                                              // split mode: tile whose partial sums are in `acc`
+            float sc[kMaxTpu], sc_next[kMaxTpu];
+#pragma unroll
+            for (int k = 0; k < kMaxTpu; ++k) {
+                sc[k] = 0.f;
+                const int tn = warp * G.tpu + k;                         // tile mode: the first unit's tiles
+                sc_next[k] = (!pl.split && k < G.tpu && tn < T) ? load_scales((long long)(t_lo + tn) * 16) : 0.f;
+            }
+            // split mode: the partial sums of tile `cur` go to its accumulator in shared memory; the warp that brings the
+            // last of a tile's contributions finishes it (returns true for that warp, with the sums in acc[0])
+            auto flush = [&]() -> bool {
+                fold(acc);
+                const int ts = (split_tiles + cur) % kTileSlots;
+                if (t < 3) {
+                    atomicAdd(&s_tile[ts][g][2 * t], acc[0][0]);
+                    atomicAdd(&s_tile[ts][g + 8][2 * t], acc[0][2]);
+                    if (t < 2) { atomicAdd(&s_tile[ts][g][2 * t + 1], acc[0][1]); atomicAdd(&s_tile[ts][g + 8][2 * t + 1], acc[0][3]); }
+                }
+                __threadfence_block();
+                __syncwarp();
+                int prev = 0;
+                if (lane == 0) prev = atomicAdd(&s_tile_cnt[ts], 1);
+                prev = __shfl_sync(0xffffffffu, prev, 0);
+                if (prev != contributors - 1) return false;
+                __threadfence_block();                                 // last to arrive: every other contribution is visible
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[0][i] = 0;
+                if (t < 3) {
+                    acc[0][0] = s_tile[ts][g][2 * t];      acc[0][2] = s_tile[ts][g + 8][2 * t];
+                    if (t < 2) { acc[0][1] = s_tile[ts][g][2 * t + 1];  acc[0][3] = s_tile[ts][g + 8][2 * t + 1]; }
+                }
+                __syncwarp();
+                if (t < 3) {                                           // leave the slot clean for the tile that reuses it
+                    s_tile[ts][g][2 * t] = 0;  s_tile[ts][g + 8][2 * t] = 0;
+                    if (t < 2) { s_tile[ts][g][2 * t + 1] = 0;  s_tile[ts][g + 8][2 * t + 1] = 0; }
+                }
+                if (lane == 0) s_tile_cnt[ts] = 0;
+                return true;
+            };
+            // unit s = warp, warp + W, ... without divisions in the loop: (tile, panel) and (stage, phase) move by fixed steps
+            const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
+            int tj = pl.split ? warp / G.n_panels : warp * G.tpu;        // first tile of the unit (relative to t_lo)
+            int pn = pl.split ? warp % G.n_panels : 0;                    // its panel
+            int slot = (it0 + warp) % P.slots;
+            uint32_t parity = (uint32_t)(((it0 + warp) / P.slots) & 1);
+            for (int s = warp; s < pl.n_units; s += W) {
+                const int n_tiles = tj < T ? min(G.tpu, T - tj) : 0;     // 0: an empty unit (padding)
+                long long fin_row0 = -1;                                 // a tile to finish after this unit, and its scales
+                float fin_sc = 0.f;
+                if (pl.split) {
+                    if (n_tiles && tj != cur) {
+                        if (cur >= 0 && flush()) { fin_row0 = (long long)(t_lo + cur) * 16; fin_sc = sc[0]; }
+                        if (fin_row0 >= 0) finish_tile(c, fin_row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], fin_sc, lane, !*abort_flag);
+                        fin_row0 = -1;
+                        cur = tj;
+                        sc[0] = load_scales((long long)(t_lo + tj) * 16);
+                        zero_acc(acc);
+                    }
+                } else if (pn == 0) {
+#pragma unroll
+                    for (int k = 0; k < kMaxTpu; ++k) {
+                        sc[k] = sc_next[k];
+                        const int tn = tj + W * G.tpu + k;                  // the same warp's next group of tiles, a round ahead
+                        if (k < G.tpu && tn < T) sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
+                    }
+                    zero_acc(acc);
+                }
+                const bool landed = wait_phase(smem_u32(&s_full[slot]), parity, abort_flag, P.wait_cycles);
+                const unsigned char* rows = ring + (size_t)slot * P.slot_bytes;
+                const bool tile_done = !pl.split && pn == G.n_panels - 1;
+                for (int k = 0; k < n_tiles; ++k) {
+                    if (k > 0) zero_acc(acc);
+                    if (landed) multiply(rows + (size_t)k * 16 * G.stride, pn, acc);
+                    if (k == n_tiles - 1) {                               // the last read of the stage is done
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+                    }
+                    if (tile_done) {
+                        fold(acc);
+                        finish_tile(c, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
+                                    k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3], lane, !*abort_flag);
+                    }
+                }
+                if (n_tiles == 0) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
+                }
+                // next unit of this warp
+                if (pl.split) {
+                    tj += step_t; pn += step_p;
+                    if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
+                } else if (++pn == G.n_panels) { pn = 0; tj += W * G.tpu; }
+                slot += W;
+                if (slot >= P.slots) { slot -= P.slots; parity ^= 1u; }
+            }
+            if (pl.split) {
+                if (cur >= 0 && flush())
+                    finish_tile(c, (long long)(t_lo + cur) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3], sc[0], lane, !*abort_flag);
+                split_tiles += T;
+            }
+            it0 += pl.n_units;
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && s_abort) report(P.dev_status, MATQ_ERR_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Host side
+
+struct HostProblem {
+    const uint8_t* packed;
+    int64_t N, K;
+    int r;
+    const float* alpha;
+    const float* zero;
+    const int32_t* ovf_row_ptr;
+    const uint16_t* ovf_col;
+    const void* x;
+    float* y;
+};
+
+inline size_t xs_bytes_of(const Geo& g, int r) { return (size_t)g.n_qc * ((128 / r) / 16) * 256; }
+inline int slot_bytes_of(const Geo& g) { return (16 * g.tpu * g.stride + 64 + 127) / 128 * 128; }   // a half-full last chunk is read 32 bytes past its row
+
+// Consumer warps for a list whose largest problem stages `xs_bytes` of activations and needs `slot_bytes` per stage:
+// as many as have a stage each (at most kMaxW); fewer than kMinW means the list does not fit this kernel.
+constexpr int kMinW = 4;
+inline int warps_for(size_t xs_bytes, int slot_bytes) {
+    const long long fit = ((long long)kSmemLimit - kStaticReserve - (long long)xs_bytes) / slot_bytes;
+    return (int)std::min<long long>(kMaxW, fit);
+}
+
+// Whether a problem can take this path at all (B = 1 is implied).
+inline bool eligible(int64_t N, int64_t K, int r) {
+    if (!(r == 8 || r == 4 || r == 2) || K % 128 != 0 || K > imma::kMaxK || N <= 0 || N >= (1ll << 31) - 16) return false;
+    const Geo g = geometry((int)N, (int)K, r);
+    return warps_for(xs_bytes_of(g, r), slot_bytes_of(g)) >= kMinW;
+}
+
+// Opt in once per device and kernel to the largest dynamic shared memory size the kernel may use.
+template <typename Kern>
+inline bool allow_max_smem(Kern kern, std::atomic<unsigned long long>& done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticReserve) != cudaSuccess) return false;
+    done.fetch_or(bit, std::memory_order_release);
+    return true;
+}
+
+// Tensor map over a plane as [N][row_bytes / 8] 64-bit words with a box of 16 rows x one panel.
+inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, const Geo& g) {
+    t5::EncodeTiledFn fn = t5::encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)(g.row_bytes / 8), (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)g.row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(g.stride / 8), 16u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint8_t*>(packed), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NP>
+inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, int32_t* dev_status, cudaStream_t s) {
+    static std::atomic<unsigned long long> smem_ok{0};
+    Params<NP> P;
+    long long items = 0, tiles = 0;
+    size_t xs_bytes = 0;
+    int slot_bytes = 0;
+    int m = 0;
+    for (int i = 0; i < n; ++i) {
+        if (hp[i].N == 0) continue;
+        if (!eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;
+        Problem& q = P.p[m];
+        q.packed = hp[i].packed; q.alpha = hp[i].alpha; q.zero = hp[i].zero;
+        q.ovf_row_ptr = hp[i].ovf_row_ptr; q.ovf_col = hp[i].ovf_col;
+        q.x = static_cast<const __nv_bfloat16*>(hp[i].x); q.y = hp[i].y;
+        q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.pad_ = 0;
+        q.item0 = items;
+        const Geo g = geometry(q.N, q.K, q.r);
+        if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
+        items += (long long)g.tiles * g.n_qc;
+        tiles += g.tiles;
+        xs_bytes = std::max(xs_bytes, xs_bytes_of(g, q.r));
+        slot_bytes = std::max(slot_bytes, slot_bytes_of(g));
+        ++m;
+    }
+    if (m == 0) return MATQ_OK;
+    for (int i = m; i < NP; ++i) P.p[i] = Problem{};
+    const int sms = sm_count();
+    const int grid = (int)std::min<long long>(sms, tiles);
+    const int W = warps_for(xs_bytes, slot_bytes);
+    if (W < kMinW) return MATQ_ERR_SHAPE;
+    const int fit = (int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes);
+    // Units a CTA issues: a single problem's share is known (ring no deeper than that, so that two kernels of a
+    // chain of programmatic dependent launches fit an SM together); a list keeps the ring as deep as it fits.
+    // The number of stages is a multiple of W: a stage always serves the same warp.
+    long long want = kMaxSlots;
+    if (m == 1) {
+        const Geo g = geometry(P.p[0].N, P.p[0].K, P.p[0].r);
+        const int T = (int)((g.tiles + grid - 1) / grid) + 1;
+        want = plan_of(g, T, W).n_units;
+    }
+    const int slots = (int)std::max<long long>(W, std::min<long long>(std::min(fit, kMaxSlots), want) / W * W);
+    P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0;
+    auto kern = gemv_stream<NP>;
+    if (!allow_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)((W + 1) * 32));
+    cfg.dynamicSmemBytes = xs_bytes + (size_t)slots * slot_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, P) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
+    return MATQ_OK;
+}
+
+// A list longer than one launch's descriptor table is served by several launches.
+inline int launch(const HostProblem* hp, int n, bool pdl, long long wait_cycles, int32_t* dev_status, cudaStream_t s) {
+    for (int i = 0; i < n; ++i)
+        if (hp[i].N != 0 && !eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;      // before anything is launched
+    if (n <= kSmallList) return launch_list<kSmallList>(hp, n, pdl, wait_cycles, dev_status, s);
+    for (int i = 0; i < n; i += kLargeList) {
+        const int st = launch_list<kLargeList>(hp + i, std::min(kLargeList, n - i), pdl, wait_cycles, dev_status, s);
+        if (st != MATQ_OK) return st;
+    }
+    return MATQ_OK;
+}
+
+}  // namespace gstream
+}  // namespace matq

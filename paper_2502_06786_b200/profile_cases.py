@@ -1,6 +1,6 @@
 """Small, self-contained invocations of each kernel for profilers (ncu wants short runs with few launches).
 
-    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemv4t|gemv2t|gemm
+    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemv4t|gemv2t|stream8|stream4|stream2|group4|group2|gemm
 
 (gemv4 / gemv2: the library's own choice at B = 1, the integer tensor kernel; a trailing t: the bf16 tensor kernel.)
 
@@ -49,6 +49,28 @@ def main(which: str) -> None:
         for _ in range(2):
             for i in range(n):
                 mq.gemv(P[i], K, r, a, a, X[i], y=Y[i], flags=flags)
+    elif which in ("stream8", "stream4", "stream2"):
+        # the persistent kernel on a plane large enough for its steady state: 65536 x 2304, one problem per launch
+        r = int(which[-1])
+        N3 = 65536
+        P = _planes(4, N3, K, r)
+        X = [torch.randn(1, K, device="cuda").to(torch.bfloat16) for _ in range(4)]
+        Y = [torch.empty(1, N3, device="cuda") for _ in range(4)]
+        a = torch.ones(N3, device="cuda")
+        for _ in range(2):
+            for i in range(4):
+                mq.gemv(P[i], K, r, a, a, X[i], y=Y[i], flags=mq.GEMV_STREAM)
+    elif which in ("group4", "group2"):
+        # twelve matrices of the Gemma-2-2B MLP stack (4 layers) in one matq_gemv_grouped call
+        r = int(which[-1])
+        shapes = [(9216, 2304), (9216, 2304), (2304, 9216)] * 4
+        P = [torch.randint(0, 256, (n_, k_ * r // 8), dtype=torch.uint8, device="cuda") for n_, k_ in shapes]
+        X = [torch.randn(k_, device="cuda").to(torch.bfloat16) for n_, k_ in shapes]
+        Y = [torch.empty(n_, device="cuda") for n_, k_ in shapes]
+        a = torch.ones(9216, device="cuda")
+        g = mq.gemv_group([(P[i], shapes[i][1], r, a[:shapes[i][0]], a[:shapes[i][0]], X[i], Y[i]) for i in range(len(shapes))])
+        for _ in range(3):
+            mq.gemv_grouped(g)
     elif which == "gemm":
         N2, K2, M2 = 14336, 4096, 1024      # the Mistral-7B matrix with a quarter of the tokens
         q = torch.randint(0, 256, (N2, K2), dtype=torch.uint8, device="cuda")
