@@ -68,9 +68,9 @@ namespace matq {
 namespace gstream {
 
 constexpr int kMaxSlots = 24;
-constexpr int kUnitBytes = 16 * 1184;        // largest unit
+constexpr int kUnitRow = 1184;                // bytes per row of the largest unit (16 rows)
 constexpr int kMaxTpu = 4;                   // tiles per unit at most
-constexpr int kMaxW = 11;                    // consumer warps (with the producer: 12 warps, 168 registers a thread)
+constexpr int kMaxW = 7;                    // consumer warps (with the producer: 12 warps, 168 registers a thread)
 constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
 constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
 constexpr int kSmallList = 8;
@@ -107,16 +107,18 @@ struct Params {
     int xs_bytes;             // staged activation bytes (largest problem)
     int W;                    // consumer warps
     int pdl;
+    int unit_row;             // bytes per row of the largest unit
 };
 
-// Shape of a problem's units.  Rows of up to 1184 bytes are staged whole: `tpu` (1 to 4) consecutive tiles are one
+// Shape of a problem's units.  Rows of up to `unit_row` (1184) bytes are staged whole: `tpu` (1 to 4) consecutive tiles are one
 // contiguous run of the plane, rows `row_bytes` apart in shared memory.  Longer rows are cut into `n_panels` panels
 // of `panel_qc` 64-byte chunks (an odd number, so that rows are an odd multiple of 64 bytes apart and the 128-bit
 // loads of a quarter warp fall into different banks; the last panel may be shorter), one tile per unit.
 struct Geo {
     int row_bytes, n_qc, tiles, n_panels, panel_qc, stride, contig, tpu;
 };
-__host__ __device__ inline Geo geometry(int N, int K, int r) {
+__host__ __device__ inline Geo geometry(int N, int K, int r, int unit_row) {
+    const int kUnitBytes = 16 * unit_row;
     Geo g;
     g.row_bytes = K / 8 * r;
     g.n_qc = (g.row_bytes + 63) / 64;
@@ -147,11 +149,13 @@ __host__ __device__ inline Geo geometry(int N, int K, int r) {
 //     (group g W + w, panel 0), (same group, panel 1), ...;
 //   fewer tiles than warps and several panels: tile-major, the panels of a tile are spread over the warps.
 struct Plan {
-    int split, n_units;
+    int split, n_units, tpu;
 };
 __host__ __device__ inline Plan plan_of(const Geo& g, int T, int W) {
     Plan pl;
-    const int Tu = (T + g.tpu - 1) / g.tpu;
+    pl.tpu = g.tpu;
+    if (T < W * pl.tpu) pl.tpu = T / W > 1 ? T / W : 1;      // a short share: one tile per unit rather than idle warps
+    const int Tu = (T + pl.tpu - 1) / pl.tpu;
     pl.split = (Tu < W && g.n_panels > 1) ? 1 : 0;
     pl.n_units = pl.split ? (T * g.n_panels + W - 1) / W * W : (Tu + W - 1) / W * g.n_panels * W;
     return pl;
@@ -215,7 +219,7 @@ __device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, 
     while (p < P.n) {
         const long long i0 = P.p[p].item0;
         if (i0 >= hi) return false;
-        const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r);
+        const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r, P.unit_row);
         const long long a = lo > i0 ? (lo - i0 + g.n_qc - 1) / g.n_qc : 0;
         const long long b = (hi - i0 + g.n_qc - 1) / g.n_qc;
         ++p;
@@ -313,77 +317,143 @@ __device__ __forceinline__ void multiply_unit(const unsigned char* wl_p, const u
 // the same exact integer.  |Y_i| < 1.25 * 2^(P + 1 - R i), so the offset that makes it a non-negative 32-bit
 // integer is 2^(P + 2 - R i); the constant column (2^(smax - R i) per byte) returns sum_i A_i 2^(smax - R i), which
 // removes sum_i A_i 2^(P + 2 - R i) exactly.
+constexpr int kHeld = 4;     // staging items (16 activations each) a thread keeps in registers between the two passes
+
+// Convert one staging item (16 consecutive activations, raw bf16 pairs) and store its byte units.
 template <int R>
-__device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K, int n_qc, int xexp, uint4* xs, int ctid, int nthr) {
+__device__ __forceinline__ void stage_item(const uint32_t (&raw)[8], const float (&mult)[8 / R], uint4* dst) {
+    constexpr int kF = 8 / R;                                  // fields per byte
+    int V[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float xf = (i & 1) ? bf_hi(raw[i >> 1]) : bf_lo(raw[i >> 1]);
+        V[i] = __float2int_rn(xf * mult[i % kF]);
+    }
+    uint32_t v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const int cls = i % kF;                              // 16 consecutive activations start at a byte boundary
+        const int y = cls == kF - 1 ? V[i] : V[i] - V[i + 1 < 16 ? i + 1 : i];
+        v[i] = (uint32_t)y + (1u << (imma::kP + 2 - R * cls));
+    }
+    uint32_t col[imma::kBytes][4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const uint32_t e0 = v[imma::unit_src<R>(4 * w)], e1 = v[imma::unit_src<R>(4 * w + 1)];
+        const uint32_t e2 = v[imma::unit_src<R>(4 * w + 2)], e3 = v[imma::unit_src<R>(4 * w + 3)];
+        const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e2, e3, 0x5140);
+        const uint32_t t2 = __byte_perm(e0, e1, 0x7362), t3 = __byte_perm(e2, e3, 0x7362);
+        col[0][w] = __byte_perm(t0, t1, 0x5410);  col[1][w] = __byte_perm(t0, t1, 0x7632);
+        col[2][w] = __byte_perm(t2, t3, 0x5410);  col[3][w] = __byte_perm(t2, t3, 0x7632);
+    }
+#pragma unroll
+    for (int d = 0; d < imma::kBytes; ++d) dst[4 * d] = make_uint4(col[d][0], col[d][1], col[d][2], col[d][3]);
+}
+
+// Stages the activations of one problem: every thread of the W consumer warps reads its items ONCE (the first
+// kHeld of them stay in registers across the reduction), the largest magnitude and the fp32 sum are reduced over the
+// CTA, then the items are converted and stored.  Two named barriers; the first also separates the previous
+// problem's multiplies from the restaging.  Returns the sum of x and the biased exponent of max |x|.
+template <int R>
+__device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K, int n_qc, uint4* xs, int ctid, int nthr, int W,
+                                                  uint32_t* s_rmax, float* s_rsum, float& xsum_out, int& xexp_out) {
     constexpr int kWpp = 128 / R;
     constexpr int kM2 = kWpp / 16;
-    constexpr int kF = 8 / R;                                  // fields per byte
+    constexpr int kF = 8 / R;
+    const int lane = ctid & 31, warp = ctid >> 5;
+    const int n_items = n_qc * kM2 * 4;
+    auto k0_of = [&](int it) {
+        const int tt = it & 3, qm = it >> 2;
+        return ((qm / kM2) * 4 + tt) * kWpp + (qm % kM2) * 16;
+    };
+    uint4 held[kHeld][2];
+    uint32_t xmax = 0;
+    float xsum = 0.f;
+    auto fold = [&](const uint4& v) {
+        xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
+        xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
+        xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
+    };
+#pragma unroll
+    for (int j = 0; j < kHeld; ++j) {
+        const int it = ctid + j * nthr;
+        const int k0 = it < n_items ? k0_of(it) : K;
+        held[j][0] = held[j][1] = make_uint4(0, 0, 0, 0);
+        if (k0 < K) { held[j][0] = ld_x4(x + k0); held[j][1] = ld_x4(x + k0 + 8); }
+    }
+#pragma unroll
+    for (int j = 0; j < kHeld; ++j) { fold(held[j][0]); fold(held[j][1]); }
+    for (int it = ctid + kHeld * nthr; it < n_items; it += nthr) {       // rows too long to hold: read again below
+        const int k0 = k0_of(it);
+        if (k0 < K) { fold(ld_x4(x + k0)); fold(ld_x4(x + k0 + 8)); }
+    }
+    xmax = max(xmax & 0xffffu, xmax >> 16);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+    }
+    if (lane == 0) { s_rmax[warp] = xmax; s_rsum[warp] = xsum; }
+    asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+    xmax = lane < W ? s_rmax[lane] : 0u;
+    xsum = lane < W ? s_rsum[lane] : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+    }
+    xsum_out = xsum;
+    const int xexp = min(max((int)(xmax >> 7), imma::kP + 1), 254);
+    xexp_out = xexp;
     float mult[kF];
 #pragma unroll
     for (int cls = 0; cls < kF; ++cls) mult[cls] = __uint_as_float((uint32_t)(254 + imma::kP - xexp - R * cls) << 23);
-    const int n_items = n_qc * kM2 * 4;
-    for (int it = ctid; it < n_items; it += nthr) {
-        const int tt = it & 3;
-        const int qm = it >> 2;
-        const int ql = qm / kM2, m2 = qm % kM2;
-        const int k0 = (ql * 4 + tt) * kWpp + m2 * 16;
-        uint32_t col[imma::kBytes][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
+#pragma unroll
+    for (int j = 0; j < kHeld; ++j) {
+        const int it = ctid + j * nthr;
+        if (it < n_items) {
+            uint4* dst = xs + (size_t)(it >> 2) * imma::kBytes * 4 + (it & 3);
+            if (k0_of(it) < K) {
+                const uint32_t raw[8] = {held[j][0].x, held[j][0].y, held[j][0].z, held[j][0].w, held[j][1].x, held[j][1].y, held[j][1].z, held[j][1].w};
+                stage_item<R>(raw, mult, dst);
+            } else {
+#pragma unroll
+                for (int d = 0; d < imma::kBytes; ++d) dst[4 * d] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
+    for (int it = ctid + kHeld * nthr; it < n_items; it += nthr) {
+        uint4* dst = xs + (size_t)(it >> 2) * imma::kBytes * 4 + (it & 3);
+        const int k0 = k0_of(it);
         if (k0 < K) {
             const uint4 va = ld_x4(x + k0), vb = ld_x4(x + k0 + 8);
             const uint32_t raw[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
-            int V[16];
+            stage_item<R>(raw, mult, dst);
+        } else {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float xf = (i & 1) ? bf_hi(raw[i >> 1]) : bf_lo(raw[i >> 1]);
-                V[i] = __float2int_rn(xf * mult[i % kF]);
-            }
-            uint32_t v[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int cls = i % kF;                          // 16 consecutive activations start at a byte boundary
-                const int y = cls == kF - 1 ? V[i] : V[i] - V[i + 1 < 16 ? i + 1 : i];
-                v[i] = (uint32_t)y + (1u << (imma::kP + 2 - R * cls));
-            }
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                const uint32_t e0 = v[imma::unit_src<R>(4 * w)], e1 = v[imma::unit_src<R>(4 * w + 1)];
-                const uint32_t e2 = v[imma::unit_src<R>(4 * w + 2)], e3 = v[imma::unit_src<R>(4 * w + 3)];
-                const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e2, e3, 0x5140);
-                const uint32_t t2 = __byte_perm(e0, e1, 0x7362), t3 = __byte_perm(e2, e3, 0x7362);
-                col[0][w] = __byte_perm(t0, t1, 0x5410);  col[1][w] = __byte_perm(t0, t1, 0x7632);
-                col[2][w] = __byte_perm(t2, t3, 0x5410);  col[3][w] = __byte_perm(t2, t3, 0x7632);
-            }
+            for (int d = 0; d < imma::kBytes; ++d) dst[4 * d] = make_uint4(0, 0, 0, 0);
         }
-        uint4* dst = xs + (size_t)qm * imma::kBytes * 4 + tt;
-#pragma unroll
-        for (int d = 0; d < imma::kBytes; ++d) dst[4 * d] = make_uint4(col[d][0], col[d][1], col[d][2], col[d][3]);
     }
+    asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
 }
-
-// What a consumer warp knows about the problem it is multiplying.
-struct Ctx {
-    const Problem* pr;
-    Geo G;
-    float xsum;
-    int xexp;
-    int sh;
-};
 
 // Finishes one tile.  Accumulator a_i of thread (g, t) holds row g + 8 (i >> 1), column 2t + (i & 1); the five
 // columns of a row are recombined in 64 bits by the lanes t = 0 and scaled back once.  `scales`: alpha of row
-// (lane) in lanes 0-15, zero of row (lane - 16) in lanes 16-31.  Called by whole warps.
-__device__ __noinline__ void finish_tile(const Ctx& c, long long row0, int a0, int a1, int a2, int a3, float scales, int lane, bool store) {
+// (lane) in lanes 0-15, zero of row (lane - 16) in lanes 16-31.  Called by whole warps.  Everything is passed by
+// value: a structure would live in local memory, and its first load would cost a trip to the L2 per launch.
+__device__ __noinline__ void finish_tile(float* __restrict__ y, const int32_t* __restrict__ ovf_row_ptr, const uint16_t* __restrict__ ovf_col,
+                                         const __nv_bfloat16* x, int N, int sh, int xexp, float xsum, long long row0,
+                                         int a0, int a1, int a2, int a3, float scales, int lane, bool store) {
     const int g = lane >> 2, t = lane & 3;
-    const Problem& pr = *c.pr;
     // extra precision (Eq. 8): sum of the activations at the listed columns of each of the 16 rows
     float ep_lo = 0.f, ep_hi = 0.f;
-    if (pr.ovf_row_ptr) {
+    if (ovf_row_ptr) {
         for (int rl = 0; rl < 16; ++rl) {
             const long long row = row0 + rl;
             float ev = 0.f;
-            if (row < pr.N) {
-                const int e0 = pr.ovf_row_ptr[row], e1 = pr.ovf_row_ptr[row + 1];
-                for (int e = e0 + lane; e < e1; e += 32) ev += __bfloat162float(pr.x[pr.ovf_col[e]]);
+            if (row < N) {
+                const int e0 = ovf_row_ptr[row], e1 = ovf_row_ptr[row + 1];
+                for (int e = e0 + lane; e < e1; e += 32) ev += __bfloat162float(x[ovf_col[e]]);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
@@ -398,12 +468,12 @@ __device__ __noinline__ void finish_tile(const Ctx& c, long long row0, int a0, i
         const int d4 = __shfl_down_sync(0xffffffffu, d0, 2);
         const float al = __shfl_sync(0xffffffffu, scales, g + 8 * h), ze = __shfl_sync(0xffffffffu, scales, 16 + g + 8 * h);
         const long long row = row0 + g + 8 * h;
-        if (t != 0 || row >= pr.N || !store) continue;
+        if (t != 0 || row >= N || !store) continue;
         // sum_i A_i Y_i = sum_d 256^d D_d - sum_i A_i 2^(P + 2 - R i), and column 4 holds sum_i A_i 2^(sh - R i)
-        const long long tot = (((long long)d3 * 256 + d2) * 256 + d1) * 256 + d0 - ((long long)d4 << (imma::kP + 2 - c.sh));
-        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(c.xexp - imma::kP) << 23);
+        const long long tot = (((long long)d3 * 256 + d2) * 256 + d1) * 256 + d0 - ((long long)d4 << (imma::kP + 2 - sh));
+        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp - imma::kP) << 23);
         v += h ? ep_hi : ep_lo;
-        pr.y[row] = al * (v * (float)(1 << c.sh) - ze * c.xsum);
+        y[row] = al * (v * (float)(1 << sh) - ze * xsum);
     }
 }
 
@@ -425,12 +495,10 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
     unsigned char* ring = smem_raw + P.xs_bytes;
     volatile int* abort_flag = &s_abort;
 
-    if (tid == 0) {
-        s_abort = 0;
-        for (int s = 0; s < P.slots; ++s) {
-            mbar_init(smem_u32(&s_full[s]), 1);
-            mbar_init(smem_u32(&s_empty[s]), 1);
-        }
+    if (tid == 0) s_abort = 0;
+    if (tid < P.slots) {
+        mbar_init(smem_u32(&s_full[tid]), 1);
+        mbar_init(smem_u32(&s_empty[tid]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kTileSlots * 16 * imma::kCols; i += blockDim.x) (&s_tile[0][0][0])[i] = 0;
@@ -459,14 +527,14 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         int last_it = -1;                                     // latest unit this lane issued a copy for
         while (ok && next_segment(P, lo, hi, p, t_lo, t_hi)) {
             const Problem& pr = P.p[p - 1];
-            const Geo G = geometry(pr.N, pr.K, pr.r);
+            const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row);
             const int T = t_hi - t_lo;
             const Plan pl = plan_of(G, T, W);
             // Lane l feeds warp l: its units are l, l + W, ...; (tile, panel) and (stage, phase) move by fixed steps.  The
             // lanes advance independently: each probes ITS stage (without suspending) and issues its next copy as soon as
             // its warp has released the stage, so a slow consumer warp never holds back the copies of the others.
             const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
-            int tj = pl.split ? lane / G.n_panels : lane * G.tpu;
+            int tj = pl.split ? lane / G.n_panels : lane * pl.tpu;
             int pn = pl.split ? lane % G.n_panels : 0;
             int slot = (it0 + lane) % P.slots;
             int use = (it0 + lane) / P.slots;                      // how often the stage has been used before
@@ -489,7 +557,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     } else if (G.contig) {
                         // the unit is one run of the plane; rows past the end of the matrix are not fetched
                         const long long row0 = (long long)(t_lo + tj) * 16;
-                        const long long rows = min((long long)min(G.tpu, T - tj) * 16, pr.N - row0);
+                        const long long rows = min((long long)min(pl.tpu, T - tj) * 16, pr.N - row0);
                         const uint32_t bytes = (uint32_t)rows * (uint32_t)G.row_bytes;
                         mbar_arrive_expect_tx(bar, bytes);
                         bulk_g2s(dst, pr.packed + row0 * G.row_bytes, bytes, bar);
@@ -502,7 +570,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     if (pl.split) {
                         tj += step_t; pn += step_p;
                         if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
-                    } else if (++pn == G.n_panels) { pn = 0; tj += W * G.tpu; }
+                    } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
                     slot += W;
                     if (slot >= P.slots) { slot -= P.slots; ++use; }
                     s += W;
@@ -540,50 +608,38 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         int split_tiles = 0;                                   // split-mode tiles of earlier segments (a tile's slot = its count mod kTileSlots)
         int p = p_first, t_lo, t_hi;
         bool first = true;
-        Ctx c;
+        Geo G;
+        float xsum = 0.f;
+        int xexp = 0;
         while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
             const Problem& pr = P.p[p - 1];
-            c.pr = &pr;
-            c.G = geometry(pr.N, pr.K, pr.r);
-            const Geo& G = c.G;
+            G = geometry(pr.N, pr.K, pr.r, P.unit_row);
             const int R = pr.r;
-            c.sh = kCodeBits - R;
+            const int sh = kCodeBits - R;
             const int T = t_hi - t_lo;
             const Plan pl = plan_of(G, T, W);
-            if (first && P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+            // alpha and zero of this warp's first tiles do not depend on the previous kernel: requested before anything else
+            const int tpu0 = pl.tpu;
+            float sc_first[kMaxTpu];
+#pragma unroll
+            for (int k = 0; k < kMaxTpu; ++k) {
+                const int tn = pl.split ? warp / G.n_panels : warp * tpu0 + k;      // split mode: one tile per unit
+                const long long row = (long long)(t_lo + tn) * 16 + (lane & 15);
+                sc_first[k] = (k < tpu0 && tn < T && row < pr.N) ? (lane < 16 ? pr.alpha[row] : pr.zero[row]) : 0.f;
+            }
+            if (first) {
+                // The activations may still be written by the previous kernel, so they are only READ after the dependency
+                // wait; pulling their lines into the L2 earlier is harmless (the L2 is the point of coherence) and takes the
+                // HBM latency of a cold vector off the critical path.
+                for (int i = ctid * 64; i < pr.K; i += nthr * 64) asm volatile("prefetch.global.L2 [%0];" ::"l"(pr.x + i));
+                if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+            }
             first = false;
 
-            // ---- largest magnitude and fp32 sum of the activations, then their bytes in fragment order.
-            // The first barrier also separates the previous problem's multiplies from the restaging.
-            uint32_t xmax = 0;
-            float xsum = 0.f;
-            for (int i = ctid; i < (pr.K >> 3); i += nthr) {
-                const uint4 v = ld_x4(pr.x + 8 * i);
-                xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
-                xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
-                xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
-            }
-            xmax = max(xmax & 0xffffu, xmax >> 16);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
-                xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
-            }
-            if (lane == 0) { s_rmax[warp] = xmax; s_rsum[warp] = xsum; }
-            asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
-            xmax = lane < W ? s_rmax[lane] : 0u;
-            xsum = lane < W ? s_rsum[lane] : 0.f;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
-                xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
-            }
-            c.xsum = xsum;
-            c.xexp = min(max((int)(xmax >> 7), imma::kP + 1), 254);
-            if (R == 8) stage_activations<8>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
-            else if (R == 4) stage_activations<4>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
-            else stage_activations<2>(pr.x, pr.K, G.n_qc, c.xexp, xs, ctid, nthr);
-            asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+            // ---- the activations of this problem as byte units in fragment order (all consumer warps together)
+            if (R == 8) stage_activations<8>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
+            else if (R == 4) stage_activations<4>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
+            else stage_activations<2>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
 
             const int kM2 = (128 / R) / 16;
             // this lane's B source: chunk q of byte column g starts at xs[q * kM2 * 16 + g * 4 + t]; the lanes g = 4 hold
@@ -647,11 +703,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             int cur = -1;                                              // split mode: tile whose partial sums are in `acc`
             float sc[kMaxTpu], sc_next[kMaxTpu];
 #pragma unroll
-            for (int k = 0; k < kMaxTpu; ++k) {
-                sc[k] = 0.f;
-                const int tn = warp * G.tpu + k;                         // tile mode: the first unit's tiles
-                sc_next[k] = (!pl.split && k < G.tpu && tn < T) ? load_scales((long long)(t_lo + tn) * 16) : 0.f;
-            }
+            for (int k = 0; k < kMaxTpu; ++k) { sc[k] = 0.f; sc_next[k] = sc_first[k]; }      // tile mode: the first unit's tiles
             // split mode: the partial sums of tile `cur` go to its accumulator in shared memory; the warp that brings the
             // last of a tile's contributions finishes it (returns true for that warp, with the sums in acc[0])
             auto flush = [&]() -> bool {
@@ -685,29 +737,29 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             };
             // unit s = warp, warp + W, ... without divisions in the loop: (tile, panel) and (stage, phase) move by fixed steps
             const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
-            int tj = pl.split ? warp / G.n_panels : warp * G.tpu;        // first tile of the unit (relative to t_lo)
+            int tj = pl.split ? warp / G.n_panels : warp * pl.tpu;        // first tile of the unit (relative to t_lo)
             int pn = pl.split ? warp % G.n_panels : 0;                    // its panel
             int slot = (it0 + warp) % P.slots;
             uint32_t parity = (uint32_t)(((it0 + warp) / P.slots) & 1);
             for (int s = warp; s < pl.n_units; s += W) {
-                const int n_tiles = tj < T ? min(G.tpu, T - tj) : 0;     // 0: an empty unit (padding)
+                const int n_tiles = tj < T ? min(pl.tpu, T - tj) : 0;     // 0: an empty unit (padding)
                 long long fin_row0 = -1;                                 // a tile to finish after this unit, and its scales
                 float fin_sc = 0.f;
                 if (pl.split) {
                     if (n_tiles && tj != cur) {
                         if (cur >= 0 && flush()) { fin_row0 = (long long)(t_lo + cur) * 16; fin_sc = sc[0]; }
-                        if (fin_row0 >= 0) finish_tile(c, fin_row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], fin_sc, lane, !*abort_flag);
+                        if (fin_row0 >= 0) finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, fin_row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], fin_sc, lane, !*abort_flag);
                         fin_row0 = -1;
                         cur = tj;
-                        sc[0] = load_scales((long long)(t_lo + tj) * 16);
+                        sc[0] = s == warp ? sc_first[0] : load_scales((long long)(t_lo + tj) * 16);     // the first one was requested early
                         zero_acc(acc);
                     }
                 } else if (pn == 0) {
 #pragma unroll
                     for (int k = 0; k < kMaxTpu; ++k) {
                         sc[k] = sc_next[k];
-                        const int tn = tj + W * G.tpu + k;                  // the same warp's next group of tiles, a round ahead
-                        if (k < G.tpu && tn < T) sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
+                        const int tn = tj + W * pl.tpu + k;                  // the same warp's next group of tiles, a round ahead
+                        if (k < pl.tpu && tn < T) sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
                     }
                     zero_acc(acc);
                 }
@@ -723,8 +775,8 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     }
                     if (tile_done) {
                         fold(acc);
-                        finish_tile(c, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
-                                    k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3], lane, !*abort_flag);
+                        finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16,
+                                    acc[0][0], acc[0][1], acc[0][2], acc[0][3], k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3], lane, !*abort_flag);
                     }
                 }
                 if (n_tiles == 0) {
@@ -735,13 +787,13 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 if (pl.split) {
                     tj += step_t; pn += step_p;
                     if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
-                } else if (++pn == G.n_panels) { pn = 0; tj += W * G.tpu; }
+                } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
                 slot += W;
                 if (slot >= P.slots) { slot -= P.slots; parity ^= 1u; }
             }
             if (pl.split) {
                 if (cur >= 0 && flush())
-                    finish_tile(c, (long long)(t_lo + cur) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3], sc[0], lane, !*abort_flag);
+                    finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, (long long)(t_lo + cur) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3], sc[0], lane, !*abort_flag);
                 split_tiles += T;
             }
             it0 += pl.n_units;
@@ -780,7 +832,7 @@ inline int warps_for(size_t xs_bytes, int slot_bytes) {
 // Whether a problem can take this path at all (B = 1 is implied).
 inline bool eligible(int64_t N, int64_t K, int r) {
     if (!(r == 8 || r == 4 || r == 2) || K % 128 != 0 || K > imma::kMaxK || N <= 0 || N >= (1ll << 31) - 16) return false;
-    const Geo g = geometry((int)N, (int)K, r);
+    const Geo g = geometry((int)N, (int)K, r, kUnitRow);
     return warps_for(xs_bytes_of(g, r), slot_bytes_of(g)) >= kMinW;
 }
 
@@ -814,45 +866,44 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     static std::atomic<unsigned long long> smem_ok{0};
     Params<NP> P;
     long long items = 0, tiles = 0;
-    size_t xs_bytes = 0;
-    int slot_bytes = 0;
-    int m = 0;
     for (int i = 0; i < n; ++i) {
         if (hp[i].N == 0) continue;
         if (!eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;
+        const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
+        items += (long long)g.tiles * g.n_qc;
+        tiles += g.tiles;
+    }
+    if (tiles == 0) return MATQ_OK;
+    const int sms = sm_count();
+    const int grid = (int)std::min<long long>(sms, tiles);
+    const int unit_row = kUnitRow;
+    size_t xs_bytes = 0;
+    int slot_bytes = 0;
+    int m = 0;
+    long long item0 = 0;
+    for (int i = 0; i < n; ++i) {
+        if (hp[i].N == 0) continue;
         Problem& q = P.p[m];
         q.packed = hp[i].packed; q.alpha = hp[i].alpha; q.zero = hp[i].zero;
         q.ovf_row_ptr = hp[i].ovf_row_ptr; q.ovf_col = hp[i].ovf_col;
         q.x = static_cast<const __nv_bfloat16*>(hp[i].x); q.y = hp[i].y;
         q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.pad_ = 0;
-        q.item0 = items;
-        const Geo g = geometry(q.N, q.K, q.r);
+        q.item0 = item0;
+        const Geo g = geometry(q.N, q.K, q.r, unit_row);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
-        items += (long long)g.tiles * g.n_qc;
-        tiles += g.tiles;
+        item0 += (long long)g.tiles * g.n_qc;
         xs_bytes = std::max(xs_bytes, xs_bytes_of(g, q.r));
         slot_bytes = std::max(slot_bytes, slot_bytes_of(g));
         ++m;
     }
-    if (m == 0) return MATQ_OK;
     for (int i = m; i < NP; ++i) P.p[i] = Problem{};
-    const int sms = sm_count();
-    const int grid = (int)std::min<long long>(sms, tiles);
     const int W = warps_for(xs_bytes, slot_bytes);
     if (W < kMinW) return MATQ_ERR_SHAPE;
     const int fit = (int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes);
-    // Units a CTA issues: a single problem's share is known (ring no deeper than that, so that two kernels of a
-    // chain of programmatic dependent launches fit an SM together); a list keeps the ring as deep as it fits.
     // The number of stages is a multiple of W: a stage always serves the same warp.
-    long long want = kMaxSlots;
-    if (m == 1) {
-        const Geo g = geometry(P.p[0].N, P.p[0].K, P.p[0].r);
-        const int T = (int)((g.tiles + grid - 1) / grid) + 1;
-        want = plan_of(g, T, W).n_units;
-    }
-    const int slots = (int)std::max<long long>(W, std::min<long long>(std::min(fit, kMaxSlots), want) / W * W);
+    const int slots = std::min(fit, kMaxSlots) / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
-    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row;
     auto kern = gemv_stream<NP>;
     if (!allow_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
