@@ -81,7 +81,11 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
         else st5 = t5::launch<2>(packed, N, K, alpha, zero, ovf_row_ptr, ovf_col, x, B, ldx, y, ldy, dev_status, pdl, s);
         if (st5 != MATQ_ERR_SHAPE) return st5;     // a K too long for one cluster's shared memory falls through
     }
-    if (path == MATQ_GEMV_STREAM) {
+    // Extra precision at B = 1: the list kernel of the persistent path (eight lanes per row, whole CTA on long lists)
+    // replaces the few threads per row of the per-matrix kernels, which take milliseconds on rows whose codes all sit
+    // in the extra bucket (heavy-tailed weights under plain min-max).
+    const bool ep_stream = path == MATQ_GEMV_AUTO && B == 1 && ovf_row_ptr && gstream::eligible(N, K, r);
+    if (path == MATQ_GEMV_STREAM || ep_stream) {
         if (B != 1 || !gstream::eligible(N, K, r)) return MATQ_ERR_SHAPE;
         const gstream::HostProblem hp = {packed, N, K, r, alpha, zero, ovf_row_ptr, ovf_col, x, y};
         return gstream::launch(&hp, 1, pdl, kStreamWaitCycles, dev_status, s);

@@ -46,8 +46,13 @@
 // nested here (see stage_activations), which saves a quarter to a half of them.
 //
 // Extra precision (Errata, Eq. 8): a listed column's field is one bucket higher
-// than the stored, clamped one, so its activation is added once more in fp32;
-// the warp that finishes a tile walks the lists of its 16 rows.
+// than the stored, clamped one, so its activation is added once more in fp32.
+// That sparse term is a matrix-vector product with the lists as a CSR pattern of
+// ones; it has nothing in common with the dense stream (two dependent
+// global-memory round trips per row, 2-byte indices, gathers), so it runs as a
+// kernel of its own (ep_rowsum: eight lanes per row, many rows in flight) that
+// leaves sum_{j in list(n)} x_j in y[n]; the persistent kernel, launched as its
+// programmatic dependent, picks the value up when it finishes row n.
 //
 // Every wait is bounded (a limit in clock cycles, about two seconds): a wait
 // that gives up sets a flag in shared memory and MATQ_ERR_TIMEOUT in
@@ -439,41 +444,139 @@ __device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K,
 
 // Finishes one tile.  Accumulator a_i of thread (g, t) holds row g + 8 (i >> 1), column 2t + (i & 1); the five
 // columns of a row are recombined in 64 bits by the lanes t = 0 and scaled back once.  `scales`: alpha of row
-// (lane) in lanes 0-15, zero of row (lane - 16) in lanes 16-31.  Called by whole warps.  Everything is passed by
-// value: a structure would live in local memory, and its first load would cost a trip to the L2 per launch.
-__device__ __noinline__ void finish_tile(float* __restrict__ y, const int32_t* __restrict__ ovf_row_ptr, const uint16_t* __restrict__ ovf_col,
-                                         const __nv_bfloat16* x, int N, int sh, int xexp, float xsum, long long row0,
-                                         int a0, int a1, int a2, int a3, float scales, int lane, bool store) {
+// (lane) in lanes 0-15, zero of row (lane - 16) in lanes 16-31; `ep_rows`: the extra-precision sum of row (lane) in
+// lanes 0-15 (zero without lists).  Called by whole warps.  Everything is passed by value: a structure would live in
+// local memory, and its first load would cost a trip to the L2 per launch.
+__device__ __noinline__ void finish_tile(float* __restrict__ y, int N, int sh, int xexp, float xsum, long long row0,
+                                         int a0, int a1, int a2, int a3, float scales, float ep_rows, int lane, bool store) {
     const int g = lane >> 2, t = lane & 3;
-    // extra precision (Eq. 8): sum of the activations at the listed columns of each of the 16 rows
-    float ep_lo = 0.f, ep_hi = 0.f;
-    if (ovf_row_ptr) {
-        for (int rl = 0; rl < 16; ++rl) {
-            const long long row = row0 + rl;
-            float ev = 0.f;
-            if (row < N) {
-                const int e0 = ovf_row_ptr[row], e1 = ovf_row_ptr[row + 1];
-                for (int e = e0 + lane; e < e1; e += 32) ev += __bfloat162float(x[ovf_col[e]]);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ev += __shfl_xor_sync(0xffffffffu, ev, o);
-            if (rl == g) ep_lo = ev;
-            if (rl == g + 8) ep_hi = ev;
-        }
-    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {                               // rows g and g + 8
         const int d0 = h ? a2 : a0, d1 = h ? a3 : a1;
         const int d2 = __shfl_down_sync(0xffffffffu, d0, 1), d3 = __shfl_down_sync(0xffffffffu, d1, 1);
         const int d4 = __shfl_down_sync(0xffffffffu, d0, 2);
         const float al = __shfl_sync(0xffffffffu, scales, g + 8 * h), ze = __shfl_sync(0xffffffffu, scales, 16 + g + 8 * h);
+        const float ep = __shfl_sync(0xffffffffu, ep_rows, g + 8 * h);
         const long long row = row0 + g + 8 * h;
         if (t != 0 || row >= N || !store) continue;
         // sum_i A_i Y_i = sum_d 256^d D_d - sum_i A_i 2^(P + 2 - R i), and column 4 holds sum_i A_i 2^(sh - R i)
         const long long tot = (((long long)d3 * 256 + d2) * 256 + d1) * 256 + d0 - ((long long)d4 << (imma::kP + 2 - sh));
-        float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp - imma::kP) << 23);
-        v += h ? ep_hi : ep_lo;
+        const float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp - imma::kP) << 23) + ep;
         y[row] = al * (v * (float)(1 << sh) - ze * xsum);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Extra precision: y[n] = sum of x over the listed columns of row n, for every problem of a list that has lists.
+
+struct EpProblem {
+    const int32_t* row_ptr;
+    const uint16_t* col;
+    const __nv_bfloat16* x;
+    float* y;
+    int N, K;
+    long long row0;           // rows of the problems before this one
+};
+template <int NP>
+struct EpParams {
+    EpProblem p[NP];
+    long long rows;           // total rows
+    int n;
+    int pdl;
+};
+constexpr int kEpThreads = 512;
+
+constexpr int kEpLongList = 512;     // lists longer than this are summed by the whole CTA
+constexpr int kEpMaxLong = 128;      // such rows a CTA remembers per problem (more are summed by their eight lanes)
+
+// Sum of x over list entries [e0, e1) taken with stride `step` from e0 + `first`: a fixed partition of the list over the
+// lanes and over four partial sums per lane.  Lists that no slice_pack produced (entries >= K) are wrapped, not trusted.
+__device__ __forceinline__ float ep_partial(const uint16_t* __restrict__ col, const __nv_bfloat16* xs, int K, int e0, int e1, int first, int step) {
+    auto xat = [&](int c) { return __bfloat162float(xs[c < K ? c : c % K]); };
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int e = e0 + first;
+    for (; e + 3 * step < e1; e += 4 * step) {
+        const int c0 = col[e], c1 = col[e + step], c2 = col[e + 2 * step], c3 = col[e + 3 * step];
+        s0 += xat(c0); s1 += xat(c1); s2 += xat(c2); s3 += xat(c3);
+    }
+    for (; e < e1; e += step) s0 += xat(col[e]);
+    return (s0 + s1) + (s2 + s3);
+}
+
+template <int NP>
+__global__ void __launch_bounds__(kEpThreads)
+ep_rowsum(const __grid_constant__ EpParams<NP> P) {
+    extern __shared__ __align__(16) unsigned char ep_smem[];
+    __shared__ int s_long[kEpMaxLong];
+    __shared__ int s_nlong;
+    __shared__ float s_wsum[kEpThreads / 32];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(ep_smem);      // the problem's activations
+    const int tid = threadIdx.x, sub = tid & 7, grp = tid >> 3;          // eight lanes per row, 2 x 64 rows per pass
+    const unsigned gmask = 0xffu << (tid & 24);
+    if (P.pdl) {
+        asm volatile("griddepcontrol.launch_dependents;");
+        asm volatile("griddepcontrol.wait;" ::: "memory");               // x may be written by the previous kernel
+    }
+    const long long lo = P.rows * blockIdx.x / gridDim.x, hi = P.rows * (blockIdx.x + 1) / gridDim.x;
+    for (int p = 0; p < P.n; ++p) {
+        const EpProblem& pr = P.p[p];
+        const long long a = lo > pr.row0 ? lo - pr.row0 : 0;
+        const long long b = hi - pr.row0 < pr.N ? hi - pr.row0 : pr.N;
+        if (a >= b) continue;
+        __syncthreads();                                                  // the previous problem's gathers are done
+        if (tid == 0) s_nlong = 0;
+        for (int i = tid; i < (pr.K >> 3); i += kEpThreads) reinterpret_cast<uint4*>(xs)[i] = ld_x4(pr.x + 8 * i);
+        __syncthreads();
+        // two rows per group and pass: their dependent loads (row_ptr, then columns, then the gathers) overlap.
+        // A row lists at most K columns: row_ptr values that say otherwise are cut short, so that every loop ends.
+        for (long long row = a + grp; row < b; row += 2 * (kEpThreads / 8)) {
+            const long long row2 = row + kEpThreads / 8;
+            const bool two = row2 < b;
+            const int e0 = max(pr.row_ptr[row], 0), e1 = min(pr.row_ptr[row + 1], e0 + pr.K);
+            const int f0 = two ? max(pr.row_ptr[row2], 0) : 0, f1 = two ? min(pr.row_ptr[row2 + 1], f0 + pr.K) : 0;
+            const bool long_a = e1 - e0 > kEpLongList, long_b = f1 - f0 > kEpLongList;
+            bool defer_a = false, defer_b = false;
+            if (long_a || long_b) {                                       // remembered for the CTA-wide pass below
+                int slot_a = kEpMaxLong, slot_b = kEpMaxLong;
+                if (sub == 0) {
+                    if (long_a) slot_a = atomicAdd(&s_nlong, 1);
+                    if (long_b) slot_b = atomicAdd(&s_nlong, 1);
+                    if (slot_a < kEpMaxLong) s_long[slot_a] = (int)(row - a);
+                    if (slot_b < kEpMaxLong) s_long[slot_b] = (int)(row2 - a);
+                }
+                slot_a = __shfl_sync(gmask, slot_a, tid & 24);
+                slot_b = __shfl_sync(gmask, slot_b, tid & 24);
+                defer_a = long_a && slot_a < kEpMaxLong;
+                defer_b = long_b && slot_b < kEpMaxLong;
+            }
+            float sa = defer_a ? 0.f : ep_partial(pr.col, xs, pr.K, e0, e1, sub, 8);
+            float sb = (!two || defer_b) ? 0.f : ep_partial(pr.col, xs, pr.K, f0, f1, sub, 8);
+            sa += __shfl_xor_sync(gmask, sa, 4);  sb += __shfl_xor_sync(gmask, sb, 4);   // the eight lanes of this group only: the
+            sa += __shfl_xor_sync(gmask, sa, 2);  sb += __shfl_xor_sync(gmask, sb, 2);   // other groups of the warp may already have
+            sa += __shfl_xor_sync(gmask, sa, 1);  sb += __shfl_xor_sync(gmask, sb, 1);   // left the loop
+            if (sub == 0) {
+                if (!defer_a) pr.y[row] = sa;
+                if (two && !defer_b) pr.y[row2] = sb;
+            }
+        }
+        __syncthreads();
+        // long lists (a row whose codes all sit in the extra bucket lists K columns): all threads on one row at a time
+        const int n_long = min(s_nlong, kEpMaxLong);
+        for (int i = 0; i < n_long; ++i) {
+            const long long row = a + s_long[i];
+            const int e0 = max(pr.row_ptr[row], 0), e1 = min(pr.row_ptr[row + 1], e0 + pr.K);
+            float v = ep_partial(pr.col, xs, pr.K, e0, e1, tid, kEpThreads);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if ((tid & 31) == 0) s_wsum[tid >> 5] = v;
+            __syncthreads();
+            if (tid == 0) {
+                float t = 0.f;
+                for (int w = 0; w < kEpThreads / 32; ++w) t += s_wsum[w];
+                pr.y[row] = t;
+            }
+            __syncthreads();
+        }
     }
 }
 
@@ -702,8 +805,22 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             const int contributors = min(G.n_panels, W);              // split mode: warps that hold a part of a tile
             int cur = -1;                                              // split mode: tile whose partial sums are in `acc`
             float sc[kMaxTpu], sc_next[kMaxTpu];
+            float epv[kMaxTpu], epv_next[kMaxTpu];                    // extra precision: the sparse term of a tile's rows (lanes 0-15)
+            const bool ep = pr.ovf_row_ptr != nullptr;
+            // the sparse term was left in y by ep_rowsum, which this kernel has waited for (plain coherent loads)
+            auto load_ep = [&](long long row0) -> float {
+                const long long row = row0 + lane;
+                float v = 0.f;
+                if (lane < 16 && row < pr.N) asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(pr.y + row) : "memory");
+                return v;
+            };
 #pragma unroll
-            for (int k = 0; k < kMaxTpu; ++k) { sc[k] = 0.f; sc_next[k] = sc_first[k]; }      // tile mode: the first unit's tiles
+            for (int k = 0; k < kMaxTpu; ++k) {
+                sc[k] = 0.f; sc_next[k] = sc_first[k];                      // tile mode: the first unit's tiles
+                epv[k] = 0.f;
+                const int tn = warp * pl.tpu + k;
+                epv_next[k] = (ep && !pl.split && k < pl.tpu && tn < T) ? load_ep((long long)(t_lo + tn) * 16) : 0.f;
+            }
             // split mode: the partial sums of tile `cur` go to its accumulator in shared memory; the warp that brings the
             // last of a tile's contributions finishes it (returns true for that warp, with the sums in acc[0])
             auto flush = [&]() -> bool {
@@ -741,15 +858,16 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             int pn = pl.split ? warp % G.n_panels : 0;                    // its panel
             int slot = (it0 + warp) % P.slots;
             uint32_t parity = (uint32_t)(((it0 + warp) / P.slots) & 1);
+            // split mode: the warp that completes a tile finishes it
+            auto finish_split = [&](long long row0, float scales) {
+                const float ep_rows = ep ? load_ep(row0) : 0.f;
+                finish_tile(pr.y, pr.N, sh, xexp, xsum, row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], scales, ep_rows, lane, !*abort_flag);
+            };
             for (int s = warp; s < pl.n_units; s += W) {
                 const int n_tiles = tj < T ? min(pl.tpu, T - tj) : 0;     // 0: an empty unit (padding)
-                long long fin_row0 = -1;                                 // a tile to finish after this unit, and its scales
-                float fin_sc = 0.f;
                 if (pl.split) {
                     if (n_tiles && tj != cur) {
-                        if (cur >= 0 && flush()) { fin_row0 = (long long)(t_lo + cur) * 16; fin_sc = sc[0]; }
-                        if (fin_row0 >= 0) finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, fin_row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], fin_sc, lane, !*abort_flag);
-                        fin_row0 = -1;
+                        if (cur >= 0 && flush()) finish_split((long long)(t_lo + cur) * 16, sc[0]);
                         cur = tj;
                         sc[0] = s == warp ? sc_first[0] : load_scales((long long)(t_lo + tj) * 16);     // the first one was requested early
                         zero_acc(acc);
@@ -758,8 +876,12 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
 #pragma unroll
                     for (int k = 0; k < kMaxTpu; ++k) {
                         sc[k] = sc_next[k];
+                        epv[k] = epv_next[k];
                         const int tn = tj + W * pl.tpu + k;                  // the same warp's next group of tiles, a round ahead
-                        if (k < pl.tpu && tn < T) sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
+                        if (k < pl.tpu && tn < T) {
+                            sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
+                            if (ep) epv_next[k] = load_ep((long long)(t_lo + tn) * 16);
+                        }
                     }
                     zero_acc(acc);
                 }
@@ -775,8 +897,9 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     }
                     if (tile_done) {
                         fold(acc);
-                        finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16,
-                                    acc[0][0], acc[0][1], acc[0][2], acc[0][3], k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3], lane, !*abort_flag);
+                        finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
+                                    k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3],
+                                    k == 0 ? epv[0] : k == 1 ? epv[1] : k == 2 ? epv[2] : epv[3], lane, !*abort_flag);
                     }
                 }
                 if (n_tiles == 0) {
@@ -792,8 +915,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 if (slot >= P.slots) { slot -= P.slots; parity ^= 1u; }
             }
             if (pl.split) {
-                if (cur >= 0 && flush())
-                    finish_tile(pr.y, pr.ovf_row_ptr, pr.ovf_col, pr.x, pr.N, sh, xexp, xsum, (long long)(t_lo + cur) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3], sc[0], lane, !*abort_flag);
+                if (cur >= 0 && flush()) finish_split((long long)(t_lo + cur) * 16, sc[0]);
                 split_tiles += T;
             }
             it0 += pl.n_units;
@@ -902,6 +1024,45 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     const int fit = (int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes);
     // The number of stages is a multiple of W: a stage always serves the same warp.
     const int slots = std::min(fit, kMaxSlots) / W * W;
+    // Extra precision: the sparse term of every problem with lists goes to its y first (see ep_rowsum); the persistent
+    // kernel then runs as that kernel's programmatic dependent (it touches y only after its dependency wait).
+    {
+        static std::atomic<unsigned long long> ep_smem_ok{0};
+        EpParams<NP> E;
+        long long rows = 0;
+        int me = 0, k_max = 0;
+        for (int i = 0; i < m; ++i) {
+            const Problem& q = P.p[i];
+            if (!q.ovf_row_ptr) continue;
+            E.p[me++] = EpProblem{q.ovf_row_ptr, q.ovf_col, q.x, q.y, q.N, q.K, rows};
+            rows += q.N;
+            k_max = std::max(k_max, q.K);
+        }
+        if (me > 0) {
+            for (int i = me; i < NP; ++i) E.p[i] = EpProblem{};
+            E.rows = rows; E.n = me; E.pdl = pdl ? 1 : 0;
+            auto ek = ep_rowsum<NP>;
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess) return MATQ_ERR_CUDA;
+            const unsigned long long bit = 1ull << (dev & 63);
+            if (!(ep_smem_ok.load(std::memory_order_acquire) & bit)) {
+                if (cudaFuncSetAttribute(ek, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * (int)imma::kMaxK) != cudaSuccess) return MATQ_ERR_CUDA;
+                ep_smem_ok.fetch_or(bit, std::memory_order_release);
+            }
+            cudaLaunchConfig_t ec = {};
+            ec.gridDim = dim3((unsigned)std::max<long long>(1, std::min<long long>(4ll * sms, (rows + 63) / 64)));
+            ec.blockDim = dim3(kEpThreads);
+            ec.dynamicSmemBytes = (size_t)2 * k_max;
+            ec.stream = s;
+            cudaLaunchAttribute ea[1];
+            ea[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            ea[0].val.programmaticStreamSerializationAllowed = 1;
+            ec.attrs = ea;
+            ec.numAttrs = pdl ? 1 : 0;
+            if (cudaLaunchKernelEx(&ec, ek, E) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
+            pdl = true;
+        }
+    }
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row;
     auto kern = gemv_stream<NP>;

@@ -68,6 +68,25 @@ def test_stream_extra_precision(r, N, K):
     assert np.abs(host(y)[0] - p["y_ref"]).max() <= TOL_INT8 * rms(p["y_ref"])
 
 
+@pytest.mark.parametrize("r", [4, 2])
+def test_stream_extra_precision_full_and_empty_rows(r):
+    # rows whose every code is in the extra bucket (a list as long as the row), rows with none, a ragged last tile
+    N, K = 77, 2304
+    q = synth.skewed_codes((N, K), 0.05, 224, 4321 + r)
+    q[3, :] = 255
+    q[16:19, :] = 250
+    q[40, :] = 0
+    q[76, ::2] = 255
+    W = synth.normal_bf16((N, K), 0.02, 99)
+    _, _, a, z = ref.quantize(W)
+    x = synth.normal_bf16((1, K), 1.0, 98)
+    sp = ref.slice_pack(q, r, extra_precision=True)
+    _, y_ref = ref.gemv(sp["packed"], K, r, a, z, x, sp["ovf_row_ptr"], sp["ovf_col"])
+    y = mq.gemv(dev(sp["packed"]), K, r, dev(a), dev(z), bf16_dev(x), ovf_row_ptr=dev(sp["ovf_row_ptr"]), ovf_col=dev(sp["ovf_col"]),
+                flags=mq.GEMV_STREAM)
+    assert np.abs(host(y)[0] - y_ref[0]).max() <= TOL_INT8 * rms(y_ref[0])
+
+
 @pytest.mark.parametrize("r", [8, 4, 2])
 @pytest.mark.parametrize("kind", ["zero", "outlier", "large", "small", "one_hot"])
 def test_stream_activation_ranges(r, kind):
