@@ -10,7 +10,9 @@
  *
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers owned by the caller unless the comment says
- *     "host".  The library never allocates, frees or keeps a pointer.
+ *     "host".  The library never allocates, frees or keeps a pointer (the one
+ *     exception, entry point (5), keeps the address of its own built-in array:
+ *     see there).
  *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and
  *     the call returns without synchronising.
  *   - The return value is a status (MATQ_OK = 0).  Argument errors are found on
@@ -22,7 +24,10 @@
  *     stated per call select the vectorised kernels; other shapes are either
  *     served by slower generic kernels or rejected with MATQ_ERR_SHAPE /
  *     MATQ_ERR_ALIGNMENT as stated.
- *   - Thread-safe; no global mutable state.
+ *   - Thread-safe: calls from several host threads need no locking.  The only
+ *     state the library keeps is write-once per device (each kernel's opt-in to
+ *     its largest shared-memory size, the address of (5)'s array); (5)'s array
+ *     itself is shared by all calls of (5) on a GPU, see there.
  */
 #ifndef MATQ_H_
 #define MATQ_H_
@@ -69,6 +74,10 @@ enum matq_gemv_flags {
                                   streamed by bulk copies into a ring in shared memory; the kernel behind
                                   matq_gemv_grouped, here with a list of one */
     MATQ_GEMV_PATH_MASK = 0xff,
+    MATQ_GEMV_TEST_STALL = 0x8000, /* matq_gemv_grouped only, for testing the error path: the kernel's producer issues no
+                                  copies, so every wait for data runs out (after about a millisecond instead of two
+                                  seconds); the call then reports MATQ_ERR_TIMEOUT through dev_status, writes no output
+                                  and returns, and the next call on the same stream works as usual */
     MATQ_GEMV_PDL = 0x100      /* launch with programmatic stream serialisation: the kernel starts
                                   fetching weights (plane, alpha, zero, overflow lists) while the previous
                                   kernel in the stream drains and waits for it only before reading x.
@@ -162,7 +171,8 @@ int matq_slice_pack(const uint8_t *q, int64_t N, int64_t K, int c, int r, int ex
  *   x            in   bf16 [B, K], row stride ldx elements, 1 <= B <= 16, 16-byte aligned, ldx % 8 == 0
  *   y            out  fp32 [B, N], row stride ldy elements
  *   workspace         device scratch of at least matq_gemv_workspace_bytes(...) bytes (may be NULL if that is 0)
- *   flags             matq_gemv_flags
+ *   flags             matq_gemv_flags; 0 (MATQ_GEMV_AUTO) is the only value a caller needs, MATQ_GEMV_PDL an optimisation for
+ *                     chains of calls, the path values exist for tests and measurements
  *   Results differ from an fp64 evaluation by rounding only.  B = 1 (and K <= 32768) sums exact integer
  *   products of the fields with the activations scaled to 30-bit integers by a power of two taken from
  *   max |x| (an activation below 2^-22 of the largest is rounded to an absolute 2^-24 of the largest at worst),
@@ -193,7 +203,7 @@ int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
  *                     or both given, x bf16 [K] 16-byte aligned, y fp32 [N].  r in {8, 4, 2}, K % 128 == 0, K <= 32768.
  *                     A problem with N == 0 is skipped.  The array is read during the call only.
  *   n_problems      any number >= 0; up to 128 problems share a launch, longer lists take several
- *   flags           0 or MATQ_GEMV_PDL (meaning as for matq_gemv: no plane, alpha, zero or list of the call is
+ *   flags           0 or MATQ_GEMV_PDL (MATQ_GEMV_TEST_STALL for tests of the error path; meaning of PDL as for matq_gemv: no plane, alpha, zero or list of the call is
  *                   written by the previous kernel of the stream)
  *   A wait inside the kernel that does not end within about two seconds sets dev_status = MATQ_ERR_TIMEOUT; the
  *   outputs are then unspecified and the kernel still returns.
@@ -275,7 +285,8 @@ int matq_gemm_multi_loss(int src_kind, const void *Wsrc, int64_t N, int64_t K, i
  *   MATQ_ERR_WORKSPACE is returned, before anything is launched, when
  *     matq_gemm_multi_workspace_bytes(src_kind, M, N, K, n_r) > matq_gemm_multi_static_max_bytes().
  *   The first call on each device looks up the array's device address (that device must be current) and should be
- *   made before any stream capture begins.  All calls on a GPU share the array and it keeps the previous call's
+ *   made before any stream capture begins.  The address is kept for the life of the process: after a cudaDeviceReset
+ *   it is stale, and this entry point must not be used on that device again.  All calls on a GPU share the array and it keeps the previous call's
  *   contents; none of it needs to start at zero, but calls that overlap on the GPU race on it and must be ordered
  *   by the caller (one stream, or events between streams).
  */

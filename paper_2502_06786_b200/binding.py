@@ -20,6 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_SHAPE, ERR_ALIGNMENT = 0, 1, 2, 3, 4
 ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_CAPACITY, ERR_TIMEOUT = 5, 6, 8, 9, 10
 SRC_BF16, SRC_CODES8, SRC_PACKED = 0, 1, 2
 GEMV_AUTO, GEMV_CUDA_CORE, GEMV_TENSOR, GEMV_TCGEN05, GEMV_TENSOR_INT8, GEMV_STREAM, GEMV_PDL = 0, 1, 2, 3, 4, 5, 0x100
+GEMV_TEST_STALL = 0x8000
 TEACHER_AND_TARGET = 256    # matq_gemm_multi_loss: teacher[i] = TEACHER_AND_TARGET + j
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",

@@ -1,6 +1,8 @@
 // Shared device/host helpers of the CUDA library (sm_100a only).
 #pragma once
 
+#include <atomic>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -37,6 +39,24 @@ inline int sm_count() {
     if (cudaGetDevice(&dev) != cudaSuccess) return 148;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
     return n;
+}
+
+// Opts a kernel in, once per device, to the largest dynamic shared memory size an SM offers it (227 KB less the
+// kernel's static shared memory).  The attribute belongs to the function, not to a launch: setting it to each call's
+// size would let two host threads with different shapes undo one another between the setting and the launch.
+// `done` holds one bit per device; give every kernel (every template instance) its own.
+template <typename Kern>
+inline bool opt_in_max_smem(Kern kern, std::atomic<unsigned long long>& done) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return true;
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, kern) != cudaSuccess) { cudaGetLastError(); return false; }
+    const int max_dynamic = 227 * 1024 - (int)attr.sharedSizeBytes;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_dynamic) != cudaSuccess) { cudaGetLastError(); return false; }
+    done.fetch_or(bit, std::memory_order_release);
+    return true;
 }
 
 }  // namespace matq

@@ -581,8 +581,8 @@ static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K,
     if (stages > kMaxStages) stages = kMaxStages;
     P.stages = stages;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
-    if (cudaFuncSetAttribute(gemm_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return MATQ_ERR_CUDA;
+    static std::atomic<unsigned long long> smem_ok{0};
+    if (!matq::opt_in_max_smem(gemm_multi_kernel, smem_ok)) return MATQ_ERR_CUDA;
     const dim3 grid((unsigned)((M + kBM - 1) / kBM), (unsigned)((N + cta_n - 1) / cta_n), 1);
     gemm_multi_kernel<<<grid, kThreads, smem, s>>>(tm_x, tm_b[0], tm_b[1], tm_b[2], P);
     return launch_status();

@@ -61,13 +61,14 @@ extern "C" int matq_gemm_multi_static(int src_kind, const void* Wsrc, int64_t N,
                                       int32_t* dev_status, void* stream) {
     using namespace matq;
     if (M < 0 || N < 0 || K <= 0 || n_r < 1 || n_r > 3) return MATQ_ERR_INVALID_ARG;
-    // size check first: a problem that does not fit the built-in array is refused without touching the GPU
-    const size_t need = matq_gemm_multi_workspace_bytes(src_kind, M, N, K, n_r);
-    if (need == 0 && M > 0 && N > 0) return MATQ_ERR_INVALID_ARG;
-    if (need > kStaticScratchBytes) return MATQ_ERR_WORKSPACE;
+    // an empty problem needs no scratch, whatever N * K says: it behaves exactly like matq_gemm_multi
     if (M == 0 || N == 0)
         return matq_gemm_multi(src_kind, Wsrc, N, K, c, alpha, zero, extra_precision, ovf_row_ptr, ovf_col, X, M, ldx,
                                rs, n_r, Y, ldy, nullptr, 0, dev_status, stream);
+    // size check next: a problem that does not fit the built-in array is refused without touching the GPU
+    const size_t need = matq_gemm_multi_workspace_bytes(src_kind, M, N, K, n_r);
+    if (need == 0) return MATQ_ERR_INVALID_ARG;
+    if (need > kStaticScratchBytes) return MATQ_ERR_WORKSPACE;
     void* scratch = nullptr;
     const int st = static_scratch(&scratch);
     if (st != MATQ_OK) return st;

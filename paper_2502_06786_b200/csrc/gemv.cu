@@ -23,6 +23,7 @@ int launch_imma_split(int mt, int sk, const uint8_t* packed, int64_t N, int64_t 
 }
 
 constexpr long long kStreamWaitCycles = 4000000000ll;         // limit of its waits: about two seconds of SM clock
+constexpr long long kStallWaitCycles = 2000000ll;            // the same under MATQ_GEMV_TEST_STALL: about a millisecond
 
 }  // namespace
 
@@ -30,7 +31,8 @@ extern "C" int matq_gemv_grouped(const matq_gemv_problem* problems, int n_proble
                                  int32_t* dev_status, void* stream) {
     using namespace matq;
     if (n_problems < 0 || (n_problems > 0 && !problems)) return MATQ_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)MATQ_GEMV_PDL) return MATQ_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(MATQ_GEMV_PDL | MATQ_GEMV_TEST_STALL)) return MATQ_ERR_INVALID_ARG;
+    const bool stall = (flags & MATQ_GEMV_TEST_STALL) != 0;
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     static_assert(sizeof(gstream::HostProblem) == sizeof(matq_gemv_problem), "descriptor layouts must agree");
     for (int i = 0; i < n_problems; ++i) {
@@ -41,7 +43,8 @@ extern "C" int matq_gemv_grouped(const matq_gemv_problem* problems, int n_proble
         if (q.K % 128 != 0 || q.K > imma::kMaxK || q.N >= (1ll << 31) - 16) return MATQ_ERR_SHAPE;
         if ((q.N > 0 && !aligned16(q.packed)) || !aligned16(q.x)) return MATQ_ERR_ALIGNMENT;
     }
-    return gstream::launch(reinterpret_cast<const gstream::HostProblem*>(problems), n_problems, (flags & MATQ_GEMV_PDL) != 0, kStreamWaitCycles, dev_status, static_cast<cudaStream_t>(stream));
+    return gstream::launch(reinterpret_cast<const gstream::HostProblem*>(problems), n_problems, (flags & MATQ_GEMV_PDL) != 0,
+                           stall ? kStallWaitCycles : kStreamWaitCycles, stall, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
@@ -88,7 +91,7 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     if (path == MATQ_GEMV_STREAM || ep_stream) {
         if (B != 1 || !gstream::eligible(N, K, r)) return MATQ_ERR_SHAPE;
         const gstream::HostProblem hp = {packed, N, K, r, alpha, zero, ovf_row_ptr, ovf_col, x, y};
-        return gstream::launch(&hp, 1, pdl, kStreamWaitCycles, dev_status, s);
+        return gstream::launch(&hp, 1, pdl, kStreamWaitCycles, false, dev_status, s);
     }
     // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at ONE wave of CTAs
     // (a second, partly filled wave costs up to 40 %; measured on B200 for 4-26 MB planes):

@@ -392,8 +392,9 @@ inline int launch(const uint8_t* packed, int64_t N, int64_t K, const float* alph
     P.qc_pass = (P.n_qc + passes - 1) / passes;
     const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
     auto kern = ovf_row_ptr ? gemv_imma<R, MT, SK, WARPS, true> : gemv_imma<R, MT, SK, WARPS, false>;
+    static std::atomic<unsigned long long> smem_ok[2] = {{0}, {0}};     // one per kernel of this template instance
     if (smem > 16 * 1024 &&   // the 48 KB default counts static shared memory too
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        !opt_in_max_smem(kern, smem_ok[ovf_row_ptr ? 1 : 0]))
         return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows), 1, 1);

@@ -113,6 +113,7 @@ struct Params {
     int W;                    // consumer warps
     int pdl;
     int unit_row;             // bytes per row of the largest unit
+    int hold;                 // diagnostics: the producer issues no copies, so every wait for a stage runs out
 };
 
 // Shape of a problem's units.  Rows of up to `unit_row` (1184) bytes are staged whole: `tpu` (1 to 4) consecutive tiles are one
@@ -628,7 +629,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         int p = p_first, t_lo, t_hi;
         bool ok = true;
         int last_it = -1;                                     // latest unit this lane issued a copy for
-        while (ok && next_segment(P, lo, hi, p, t_lo, t_hi)) {
+        while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi)) {
             const Problem& pr = P.p[p - 1];
             const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row);
             const int T = t_hi - t_lo;
@@ -958,18 +959,6 @@ inline bool eligible(int64_t N, int64_t K, int r) {
     return warps_for(xs_bytes_of(g, r), slot_bytes_of(g)) >= kMinW;
 }
 
-// Opt in once per device and kernel to the largest dynamic shared memory size the kernel may use.
-template <typename Kern>
-inline bool allow_max_smem(Kern kern, std::atomic<unsigned long long>& done) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    const unsigned long long bit = 1ull << (dev & 63);
-    if (done.load(std::memory_order_acquire) & bit) return true;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticReserve) != cudaSuccess) return false;
-    done.fetch_or(bit, std::memory_order_release);
-    return true;
-}
-
 // Tensor map over a plane as [N][row_bytes / 8] 64-bit words with a box of 16 rows x one panel.
 inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, const Geo& g) {
     t5::EncodeTiledFn fn = t5::encode_fn();
@@ -984,7 +973,7 @@ inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, co
 }
 
 template <int NP>
-inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, int32_t* dev_status, cudaStream_t s) {
+inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     static std::atomic<unsigned long long> smem_ok{0};
     Params<NP> P;
     long long items = 0, tiles = 0;
@@ -1042,13 +1031,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
             for (int i = me; i < NP; ++i) E.p[i] = EpProblem{};
             E.rows = rows; E.n = me; E.pdl = pdl ? 1 : 0;
             auto ek = ep_rowsum<NP>;
-            int dev = 0;
-            if (cudaGetDevice(&dev) != cudaSuccess) return MATQ_ERR_CUDA;
-            const unsigned long long bit = 1ull << (dev & 63);
-            if (!(ep_smem_ok.load(std::memory_order_acquire) & bit)) {
-                if (cudaFuncSetAttribute(ek, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * (int)imma::kMaxK) != cudaSuccess) return MATQ_ERR_CUDA;
-                ep_smem_ok.fetch_or(bit, std::memory_order_release);
-            }
+            if (!opt_in_max_smem(ek, ep_smem_ok)) return MATQ_ERR_CUDA;
             cudaLaunchConfig_t ec = {};
             ec.gridDim = dim3((unsigned)std::max<long long>(1, std::min<long long>(4ll * sms, (rows + 63) / 64)));
             ec.blockDim = dim3(kEpThreads);
@@ -1064,9 +1047,9 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         }
     }
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
-    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
     auto kern = gemv_stream<NP>;
-    if (!allow_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
+    if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)((W + 1) * 32));
@@ -1082,12 +1065,12 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
 }
 
 // A list longer than one launch's descriptor table is served by several launches.
-inline int launch(const HostProblem* hp, int n, bool pdl, long long wait_cycles, int32_t* dev_status, cudaStream_t s) {
+inline int launch(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     for (int i = 0; i < n; ++i)
         if (hp[i].N != 0 && !eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;      // before anything is launched
-    if (n <= kSmallList) return launch_list<kSmallList>(hp, n, pdl, wait_cycles, dev_status, s);
+    if (n <= kSmallList) return launch_list<kSmallList>(hp, n, pdl, wait_cycles, hold, dev_status, s);
     for (int i = 0; i < n; i += kLargeList) {
-        const int st = launch_list<kLargeList>(hp + i, std::min(kLargeList, n - i), pdl, wait_cycles, dev_status, s);
+        const int st = launch_list<kLargeList>(hp + i, std::min(kLargeList, n - i), pdl, wait_cycles, hold, dev_status, s);
         if (st != MATQ_OK) return st;
     }
     return MATQ_OK;

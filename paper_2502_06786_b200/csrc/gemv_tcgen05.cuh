@@ -460,7 +460,8 @@ inline int launch(const uint8_t* packed, int64_t N, int64_t K, const float* alph
     // (2 x 256): tcgen05.alloc then never has to wait for another CTA.
     const size_t smem = smem_for(sb) < 80 * 1024 ? 80 * 1024 : smem_for(sb);
     auto kern = gemv_tcgen05<R>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return MATQ_ERR_CUDA;
+    static std::atomic<unsigned long long> smem_ok{0};
+    if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)row_blocks, (unsigned)n_split, 1);
     cfg.blockDim = dim3(kThreads);

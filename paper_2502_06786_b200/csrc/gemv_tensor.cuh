@@ -514,8 +514,9 @@ inline int launch_gemv_tensor(const uint8_t* packed, int64_t N, int64_t K, const
     P.qc_pass = (c_per + passes - 1) / passes;
     const size_t smem = (size_t)P.qc_pass * chunk_bytes + part_bytes;
     auto kern = ovf_row_ptr ? gemv_tensor<R, MT, NT, SK, WARPS, true, CL> : gemv_tensor<R, MT, NT, SK, WARPS, false, CL>;
+    static std::atomic<unsigned long long> smem_ok[2] = {{0}, {0}};     // one per kernel of this template instance
     if (smem > 16 * 1024 &&   // the 48 KB default counts static shared memory too
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        !opt_in_max_smem(kern, smem_ok[ovf_row_ptr ? 1 : 0]))
         return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows) * CL, 1, 1);

@@ -414,8 +414,9 @@ extern "C" int matq_quantize_clip(const void* W, int64_t N, int64_t K, int64_t l
 #undef MATQ_QUANT_REG
     } else if (fast) {
         const size_t smem = (size_t)K * 2;
+        static std::atomic<unsigned long long> smem_ok{0};
         if (smem > 40 * 1024 &&   // the 48 KB default counts static shared memory too
-            cudaFuncSetAttribute(quantize_rows_vec, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            !opt_in_max_smem(quantize_rows_vec, smem_ok))
             return MATQ_ERR_CUDA;
         int per_sm = (int)((200u * 1024u) / (smem + 1024));
         per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);

@@ -543,8 +543,9 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     if (rpw < 1) return MATQ_ERR_SHAPE;
     const int T = nwarps * rpw;
     const size_t smem = (size_t)T * row_smem;
+    static std::atomic<unsigned long long> smem_ok{0};     // one per template instance
     if (smem > 40 * 1024 &&   // the 48 KB default counts static shared memory too
-        cudaFuncSetAttribute(slice_pack_ep<PACK_R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEpSmemLimit) != cudaSuccess)
+        !opt_in_max_smem(slice_pack_ep<PACK_R>, smem_ok))
         return MATQ_ERR_CUDA;
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, slice_pack_ep<PACK_R>, nwarps * 32, smem) != cudaSuccess ||

@@ -192,3 +192,48 @@ def test_argument_errors_and_empty():
     assert call(wsb=16) == mq.ERR_WORKSPACE and call(ws=None) == mq.ERR_WORKSPACE
     assert call(M=0) == mq.OK
     assert mq.gemm_multi_workspace_bytes(mq.SRC_BF16, 128, 128, 128, 3) >= 128 * 128 * (1 + 6) + 512
+
+
+def _check_rows(Ys_dev, Yr, rows, tol=TOL):
+    """Rows `rows` of every device output against the oracle's outputs for exactly those rows of X."""
+    idx = torch.as_tensor(rows, device="cuda")
+    for yg, yr in zip(Ys_dev, Yr):
+        got = host(yg.index_select(0, idx))
+        err = np.abs(got - yr).max()
+        assert err <= tol * rms(yr), (err, rms(yr))
+
+
+def test_benchmark_shape_bf16_source_three_precisions():
+    # The co-training forward at its benchmark size (W 14336 x 4096, 4096 tokens: 32 x 112 output tiles, 64 K blocks per
+    # tile), in the configuration the benchmark times.  The oracle cannot do 1.4e12 flop in test time, so it computes a
+    # block of 128 consecutive token rows and 64 seeded random token rows (full K, all channels, all three precisions).
+    N, K, M = 14336, 4096, 4096
+    W = synth.normal_bf16((N, K), 0.02, synth.seed_for(4, 0))
+    X = synth.normal_bf16((M, K), 1.0, synth.seed_for(4, 500))
+    Ys, a, z = mq.gemm_multi(mq.SRC_BF16, bf16_dev(W), K, bf16_dev(X))
+    rng = np.random.default_rng(4096)
+    block = list(range(1920, 2048))                      # straddles nothing special: one whole token tile ...
+    block2 = list(range(4000, 4096))                     # ... and the end of the last one
+    scattered = sorted(rng.choice(M, size=64, replace=False).tolist())
+    for rows in (block, block2 + scattered):
+        st, Yr, ar, zr = ref.gemm_multi(ref.SRC_BF16, W, K, np.ascontiguousarray(X[rows]))
+        assert st == ref.OK
+        assert np.array_equal(host(a), ar) and np.array_equal(host(z), zr)
+        _check_rows(Ys, Yr, rows)
+
+
+def test_benchmark_shape_prefill_from_extra_precision_plane():
+    # configs[4] prefill: an extra-precision int2 plane with 5 % of the codes in the extra bucket, 14336 x 3584, 2048 tokens
+    N, K, M = 14336, 3584, 2048
+    q = synth.skewed_codes((N, K), 0.05, 224, synth.seed_for(5, 0))
+    sp = ref.slice_pack(q, 2, extra_precision=True, want_unpacked=False)
+    X = synth.normal_bf16((M, K), 1.0, synth.seed_for(5, 500))
+    a = np.full(N, 1e-3, np.float32); z = np.full(N, 128.0, np.float32)
+    Ys, _, _ = mq.gemm_multi(mq.SRC_PACKED, dev(sp["packed"]), K, bf16_dev(X), rs=(2,), alpha=dev(a), zero=dev(z), extra_precision=True,
+                             ovf_row_ptr=dev(sp["ovf_row_ptr"]), ovf_col=dev(sp["ovf_col"]))
+    rng = np.random.default_rng(2048)
+    rows = list(range(1024, 1152)) + sorted(rng.choice(M, size=64, replace=False).tolist())
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_PACKED, sp["packed"], K, np.ascontiguousarray(X[rows]), rs=(2,), alpha=a, zero=z,
+                                  extra_precision=True, ovf_row_ptr=sp["ovf_row_ptr"], ovf_col=sp["ovf_col"])
+    assert st == ref.OK
+    _check_rows(Ys, Yr, rows)

@@ -175,3 +175,22 @@ def test_grouped_argument_errors():
     g[0].ovf_row_ptr = g[0].alpha
     assert mq.gemv_grouped(g, raise_on_error=False) == mq.ERR_INVALID_ARG
     assert mq.gemv_grouped(mq.gemv_group([p]), flags=7, raise_on_error=False) == mq.ERR_INVALID_ARG
+
+
+def test_a_wait_that_runs_out_is_a_status_not_a_hang():
+    # MATQ_GEMV_TEST_STALL: the producer of the persistent kernel issues no copies, so the multiplying warps' waits for
+    # their stages run out.  The kernel must return, report MATQ_ERR_TIMEOUT, leave y alone, and the same context
+    # (same stream) must then serve the same list correctly.
+    hosts = [_problem(2048, 2304, 4, 11), _problem(300, 9216, 2, 12), _problem(515, 3584, 8, 13, ep=False)]
+    devs = [_to_device(p) for p in hosts]
+    status = status_word()
+    st = mq.gemv_grouped(devs, flags=mq.GEMV_TEST_STALL, dev_status=status, raise_on_error=False)
+    assert st == mq.OK                                    # the launch itself is fine: the error depends on the device
+    assert int(host(status)[0]) == mq.ERR_TIMEOUT
+    for d in devs:
+        assert bool(torch.isnan(d["y"]).all())          # nothing was stored
+    status.zero_()
+    mq.gemv_grouped(devs, dev_status=status)
+    for p, d in zip(hosts, devs):
+        assert np.abs(host(d["y"]) - p["y_ref"]).max() <= TOL_INT8 * rms(p["y_ref"])
+    assert int(host(status)[0]) == mq.OK

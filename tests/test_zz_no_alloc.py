@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import ref
 from paper_2502_06786_b200 import binding as mq
 from paper_2502_06786_b200 import synth
 from tests.util import bf16_dev, dev, host, rms
@@ -36,6 +37,11 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     assert mq.gemm_multi_static(mq.SRC_CODES8, q, K, X, got, a, z) == mq.OK
     for g, w in zip(got, want):
         assert np.abs(host(g) - host(w)).max() <= TOL * rms(host(w))
+    # and against the CPU oracle directly, not only against the other entry point
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, host(q), K, host(X.view(torch.uint16)).astype(np.uint16), alpha=host(a), zero=host(z))
+    assert st == ref.OK
+    for g, yr in zip(got, Yr):
+        assert np.abs(host(g) - yr).max() <= TOL * rms(yr)
 
     # call 2, straight after: another shape, bf16 source (quantises on the fly), two precisions
     M2, N2, K2 = 96, 264, 1024
