@@ -51,8 +51,8 @@ METRIC = "sliced int{8,4,2} GEMV HBM GB/s (% of peak); multi-precision GEMM TFLO
 # profiles/; a kernel that has changed since its capture reports traffic = null.
 NCU = {
     # matq_gemv_grouped on 12 matrices of this stack (profiles/gemv_stream_*.md): DRAM bytes / algorithmic bytes
-    "gemv_stream_ratio_r4": None,
-    "gemv_stream_ratio_r2": None,
+    "gemv_stream_ratio_r4": 1.028,
+    "gemv_stream_ratio_r2": 0.991,
     "quantize": 42780000,
 }
 CONFIG_ID = 2
@@ -461,12 +461,14 @@ def run_cuda(args, rank, world, local_rank):
     out = None
     if rank == 0:
         ach = gemv_bytes / (gemv_ms * 1e-3) / 1e9
-        ratio = NCU["gemv_stream_ratio_r4"]
+        r4x, r2x = NCU["gemv_stream_ratio_r4"], NCU["gemv_stream_ratio_r2"]
+        n_l = plan[i4][2] + plan[i2][2]
+        traffic = None if r4x is None or r2x is None else int((plan[i4][3] * r4x + plan[i2][3] * r2x) / n_l)
         roofline = dict(kernel="gemv_stream (matq_gemv_grouped: persistent integer-MMA GEMV, B = 1), r = 4 and r = 2 stages of the step",
                         bound="hbm", achieved=round(ach, 1), peak=peaks["hbm_gbs"], unit="GB/s", frac=round(ach / peaks["hbm_gbs"], 4),
-                        traffic=None if ratio is None else int(plan[i4][3] * ratio), peak_source=peaks["source"],
-                        traffic_note="DRAM bytes of the r = 4 whole-stack launch, scaled by matrices from the ncu capture of a 12-matrix call "
-                                     "(profiles/gemv_stream_cfg2.md): traffic grows in proportion to the planes read",
+                        traffic=traffic, peak_source=peaks["source"],
+                        traffic_note="DRAM bytes per launch (mean of the r = 4 and r = 2 whole-stack launches, like bytes_per_launch), scaled by "
+                                     "planes read from the ncu captures of 12-matrix calls (profiles/gemv_stream_cfg2_12_matrices.md)",
                         avg_launch_us=round(gemv_ms * 1e3 / (plan[i4][2] + plan[i2][2]), 2),
                         bytes_per_launch=gemv_bytes // (plan[i4][2] + plan[i2][2]), gemv_frac_hbm=gemv_frac)
         out = {
