@@ -12,7 +12,7 @@
 //     at tile boundaries, so SMs are balanced to within one tile whatever the
 //     shapes are, and a CTA prepares the activations only of the one to three
 //     problems its share touches;
-//   * one producer warp feeds a ring of 18.5 KB stages with ONE copy per stage
+//   * one producer warp feeds a ring of stages (up to 18.5 KB each) with ONE copy per stage
 //     (completion counted on an mbarrier).  A stage is one UNIT: rows of up to
 //     1184 bytes are staged whole, 1 to 4 consecutive 16-row tiles being one
 //     contiguous run of the plane (cp.async.bulk); longer rows are cut into K
@@ -75,7 +75,7 @@ namespace gstream {
 constexpr int kMaxSlots = 24;
 constexpr int kUnitRow = 1184;                // bytes per row of the largest unit (16 rows)
 constexpr int kMaxTpu = 4;                   // tiles per unit at most
-constexpr int kMaxW = 7;                    // consumer warps (with the producer: 12 warps, 168 registers a thread)
+constexpr int kMaxW = 8;                    // consumer warps: two per sub-partition; the producer warp is the ninth
 constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
 constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
 constexpr int kSmallList = 8;
@@ -1008,11 +1008,14 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         ++m;
     }
     for (int i = m; i < NP; ++i) P.p[i] = Problem{};
-    const int W = warps_for(xs_bytes, slot_bytes);
+    int W = warps_for(xs_bytes, slot_bytes);
     if (W < kMinW) return MATQ_ERR_SHAPE;
-    const int fit = (int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes);
-    // The number of stages is a multiple of W: a stage always serves the same warp.
-    const int slots = std::min(fit, kMaxSlots) / W * W;
+    const int fit = std::min((int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes), kMaxSlots);
+    // The number of stages is a multiple of W: a stage always serves the same warp.  Eight warps (two per
+    // sub-partition) unless seven get more stages out of the same shared memory (14 instead of 8, say): bytes in
+    // flight matter more than the eighth warp.
+    if (W == kMaxW && fit / (W - 1) * (W - 1) > fit / W * W) --W;
+    const int slots = fit / W * W;
     // Extra precision: the sparse term of every problem with lists goes to its y first (see ep_rowsum); the persistent
     // kernel then runs as that kernel's programmatic dependent (it touches y only after its dependency wait).
     {
