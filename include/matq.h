@@ -218,6 +218,7 @@ typedef struct matq_gemv_problem {
     const uint16_t *ovf_col;
     const void *x;
     float *y;
+    int64_t B;                   /* activation vectors: 0 or 1 = one (x bf16 [K], y fp32 [N]); 2 .. 16 = x bf16 [B, K], y fp32 [B, N], dense rows */
 } matq_gemv_problem;
 int matq_gemv_grouped(const matq_gemv_problem *problems, int n_problems, int c, unsigned flags,
                       int32_t *dev_status, void *stream);

@@ -34,7 +34,7 @@ class GemvProblem(C.Structure):
     """matq_gemv_problem."""
     _fields_ = [("packed", C.c_void_p), ("N", C.c_int64), ("K", C.c_int64), ("r", C.c_int),
                 ("alpha", C.c_void_p), ("zero", C.c_void_p), ("ovf_row_ptr", C.c_void_p), ("ovf_col", C.c_void_p),
-                ("x", C.c_void_p), ("y", C.c_void_p)]
+                ("x", C.c_void_p), ("y", C.c_void_p), ("B", C.c_int64)]
 
 
 class MatqError(RuntimeError):
@@ -221,6 +221,7 @@ def gemv(packed, K, r, alpha, zero, x, y=None, ovf_row_ptr=None, ovf_col=None, w
 
 def gemv_group(problems):
     """Descriptor array for gemv_grouped from dicts / tuples (packed, K, r, alpha, zero, x, y[, ovf_row_ptr, ovf_col]).
+    x [K] with y [N] is one activation vector; x [B, K] with y [B, N] (2 <= B <= 16, dense rows) a batch.
     Build it once and reuse it: it holds raw pointers, the caller keeps the tensors alive."""
     arr = (GemvProblem * len(problems))()
     for d, pr in zip(arr, problems):
@@ -230,12 +231,15 @@ def gemv_group(problems):
         rp, col = (pr[7], pr[8]) if len(pr) > 7 else (None, None)
         _dev(packed, torch.uint8, "packed", 2); _dev(x, torch.bfloat16, "x"); _dev(y, torch.float32, "y")
         _dev(alpha, torch.float32, "alpha"); _dev(zero, torch.float32, "zero")
-        if not packed.is_contiguous() or not x.is_contiguous() or not y.is_contiguous() or x.numel() != K or y.numel() != packed.shape[0]:
-            raise ValueError("packed, x [K] and y [N] must be contiguous and match the shape")
-        d.packed, d.N, d.K, d.r = packed.data_ptr(), packed.shape[0], K, r
+        N = packed.shape[0]
+        B = x.shape[0] if x.dim() == 2 and x.shape[0] > 1 else 1
+        if not packed.is_contiguous() or not x.is_contiguous() or not y.is_contiguous() or x.numel() != B * K or y.numel() != B * N:
+            raise ValueError("packed, x [K] or [B, K] and y [N] or [B, N] must be contiguous and match the shape")
+        d.packed, d.N, d.K, d.r = packed.data_ptr(), N, K, r
         d.alpha, d.zero, d.x, d.y = alpha.data_ptr(), zero.data_ptr(), x.data_ptr(), y.data_ptr()
         d.ovf_row_ptr = None if rp is None else rp.data_ptr()
         d.ovf_col = None if col is None else col.data_ptr()
+        d.B = B
     return arr
 
 

@@ -5,6 +5,7 @@
 #include "gemv_tcgen05.cuh"
 #include "gemv_imma.cuh"
 #include "gemv_stream.cuh"
+#include "gemv_stream_batch.cuh"
 
 namespace {
 
@@ -35,16 +36,41 @@ extern "C" int matq_gemv_grouped(const matq_gemv_problem* problems, int n_proble
     const bool stall = (flags & MATQ_GEMV_TEST_STALL) != 0;
     if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
     static_assert(sizeof(gstream::HostProblem) == sizeof(matq_gemv_problem), "descriptor layouts must agree");
+    bool any_batch = false;
     for (int i = 0; i < n_problems; ++i) {
         const matq_gemv_problem& q = problems[i];
-        if (q.N < 0 || q.K <= 0 || !q.x || (q.N > 0 && (!q.packed || !q.alpha || !q.zero || !q.y))) return MATQ_ERR_INVALID_ARG;
+        if (q.N < 0 || q.K <= 0 || q.B < 0 || q.B > 16 || !q.x || (q.N > 0 && (!q.packed || !q.alpha || !q.zero || !q.y))) return MATQ_ERR_INVALID_ARG;
         if ((q.ovf_row_ptr == nullptr) != (q.ovf_col == nullptr)) return MATQ_ERR_INVALID_ARG;
         if (!(q.r == 8 || q.r == 4 || q.r == 2)) return MATQ_ERR_UNSUPPORTED;
+        if (q.B > 1 && q.ovf_row_ptr) return MATQ_ERR_UNSUPPORTED;       // lists with several vectors: matq_gemv per matrix
         if (q.K % 128 != 0 || q.K > imma::kMaxK || q.N >= (1ll << 31) - 16) return MATQ_ERR_SHAPE;
+        if (q.B > 1 && q.r == 2 && q.K % 256 != 0) return MATQ_ERR_SHAPE;
         if ((q.N > 0 && !aligned16(q.packed)) || !aligned16(q.x)) return MATQ_ERR_ALIGNMENT;
+        any_batch = any_batch || q.B > 1;
     }
-    return gstream::launch(reinterpret_cast<const gstream::HostProblem*>(problems), n_problems, (flags & MATQ_GEMV_PDL) != 0,
-                           stall ? kStallWaitCycles : kStreamWaitCycles, stall, dev_status, static_cast<cudaStream_t>(stream));
+    const bool pdl = (flags & MATQ_GEMV_PDL) != 0;
+    const long long wait = stall ? kStallWaitCycles : kStreamWaitCycles;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const gstream::HostProblem* hp = reinterpret_cast<const gstream::HostProblem*>(problems);
+    if (!any_batch) return gstream::launch(hp, n_problems, pdl, wait, stall, dev_status, s);
+    // Single vectors and batches take different kernels: two sublists, in the order given (problems are independent).
+    // A batch larger than one launch can stage becomes several problems that share the plane.
+    std::vector<gstream::HostProblem> one, many;
+    std::vector<int> many_b;
+    for (int i = 0; i < n_problems; ++i) {
+        if (hp[i].B <= 1) { one.push_back(hp[i]); continue; }
+        const int st = gstream::split_batch(hp[i], one, many, many_b);
+        if (st != MATQ_OK) return st;
+    }
+    for (const gstream::HostProblem& q : one)
+        if (q.N != 0 && !gstream::eligible(q.N, q.K, q.r)) return MATQ_ERR_SHAPE;          // before anything is launched
+    for (size_t i = 0; i < many.size(); ++i)
+        if (many[i].N != 0 && !gstream::eligible_batch(many[i].N, many[i].K, many[i].r, many_b[i])) return MATQ_ERR_SHAPE;
+    if (!one.empty()) {
+        const int st = gstream::launch(one.data(), (int)one.size(), pdl, wait, stall, dev_status, s);
+        if (st != MATQ_OK) return st;
+    }
+    return gstream::launch_batch(many.data(), many_b.data(), (int)many.size(), pdl, wait, stall, dev_status, s);
 }
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
@@ -88,9 +114,22 @@ extern "C" int matq_gemv(const uint8_t* packed, int64_t N, int64_t K, int c, int
     // replaces the few threads per row of the per-matrix kernels, which take milliseconds on rows whose codes all sit
     // in the extra bucket (heavy-tailed weights under plain min-max).
     const bool ep_stream = path == MATQ_GEMV_AUTO && B == 1 && ovf_row_ptr && gstream::eligible(N, K, r);
+    if (path == MATQ_GEMV_STREAM && B > 1) {
+        // batches in the persistent kernel: dense rows of x and y, no lists, at most 8 vectors per problem
+        if (ovf_row_ptr) return MATQ_ERR_UNSUPPORTED;
+        if (ldx != K || ldy != N) return MATQ_ERR_SHAPE;
+        const gstream::HostProblem q = {packed, N, K, r, alpha, zero, nullptr, nullptr, x, y, B};
+        std::vector<gstream::HostProblem> one, many;
+        std::vector<int> many_b;
+        int st = gstream::split_batch(q, one, many, many_b);
+        if (st != MATQ_OK) return st;
+        if (!one.empty() && !gstream::eligible(N, K, r)) return MATQ_ERR_SHAPE;
+        if (!one.empty() && (st = gstream::launch(one.data(), (int)one.size(), pdl, kStreamWaitCycles, false, dev_status, s)) != MATQ_OK) return st;
+        return gstream::launch_batch(many.data(), many_b.data(), (int)many.size(), pdl || !one.empty(), kStreamWaitCycles, false, dev_status, s);
+    }
     if (path == MATQ_GEMV_STREAM || ep_stream) {
         if (B != 1 || !gstream::eligible(N, K, r)) return MATQ_ERR_SHAPE;
-        const gstream::HostProblem hp = {packed, N, K, r, alpha, zero, ovf_row_ptr, ovf_col, x, y};
+        const gstream::HostProblem hp = {packed, N, K, r, alpha, zero, ovf_row_ptr, ovf_col, x, y, 1};
         return gstream::launch(&hp, 1, pdl, kStreamWaitCycles, false, dev_status, s);
     }
     // Warp tile: 16*MT rows x K/SK; the SK warps of a row tile sit in one CTA.  The split aims at ONE wave of CTAs

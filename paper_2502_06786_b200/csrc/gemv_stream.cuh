@@ -95,7 +95,7 @@ struct Problem {
     float* y;
     int N, K;
     int r;
-    int pad_;
+    int B;                    // activation vectors (1 in gemv_stream; 2 .. 8 in gemv_stream_batch)
     long long item0;          // (tile x chunk) items of the problems before this one
 };
 
@@ -324,6 +324,7 @@ __device__ __forceinline__ void multiply_unit(const unsigned char* wl_p, const u
 // integer is 2^(P + 2 - R i); the constant column (2^(smax - R i) per byte) returns sum_i A_i 2^(smax - R i), which
 // removes sum_i A_i 2^(P + 2 - R i) exactly.
 constexpr int kHeld = 4;     // staging items (16 activations each) a thread keeps in registers between the two passes
+constexpr int kSumThreads = 128;   // threads that sum x: the smallest number of consumer threads a launch can have (kMinW warps)
 
 // Convert one staging item (16 consecutive activations, raw bf16 pairs) and store its byte units.
 template <int R>
@@ -378,7 +379,9 @@ __device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K,
     auto fold = [&](const uint4& v) {
         xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
         xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
-        xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
+    };
+    auto sum8 = [](const uint4& v) {
+        return ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
     };
 #pragma unroll
     for (int j = 0; j < kHeld; ++j) {
@@ -387,6 +390,13 @@ __device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K,
         held[j][0] = held[j][1] = make_uint4(0, 0, 0, 0);
         if (k0 < K) { held[j][0] = ld_x4(x + k0); held[j][1] = ld_x4(x + k0 + 8); }
     }
+    // The fp32 sum of x is taken by the first kSumThreads threads in an order that does not depend on the number of
+    // consumer warps, so a problem gives the same bits in every list and launch shape (the integer sums do anyway).
+    if (ctid < kSumThreads)
+        for (int it = ctid; it < n_items; it += kSumThreads) {
+            const int k0 = k0_of(it);
+            if (k0 < K) { xsum += sum8(ld_x4(x + k0)); xsum += sum8(ld_x4(x + k0 + 8)); }
+        }
 #pragma unroll
     for (int j = 0; j < kHeld; ++j) { fold(held[j][0]); fold(held[j][1]); }
     for (int it = ctid + kHeld * nthr; it < n_items; it += nthr) {       // rows too long to hold: read again below
@@ -402,7 +412,7 @@ __device__ __forceinline__ void stage_activations(const __nv_bfloat16* x, int K,
     if (lane == 0) { s_rmax[warp] = xmax; s_rsum[warp] = xsum; }
     asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
     xmax = lane < W ? s_rmax[lane] : 0u;
-    xsum = lane < W ? s_rsum[lane] : 0.f;
+    xsum = lane < kSumThreads / 32 ? s_rsum[lane] : 0.f;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
@@ -581,6 +591,94 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
     }
 }
 
+// The producer warp of a CTA: lane l < W feeds consumer warp l's stages with the units of this CTA's share [lo, hi), in
+// the order plan_of() defines.  Shared by the kernels that consume the ring.
+template <int NP>
+__device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo, long long hi, int p_first, int W, unsigned char* ring,
+                                              uint64_t* s_full, uint64_t* s_empty, volatile int* abort_flag, int lane) {
+    // ------------------------------------------------------------------ producer warp: lane l < W feeds warp l's stages
+    int it0 = 0;                                          // units of the segments before this one (a multiple of W)
+    bool waited = !P.pdl;
+    int p = p_first, t_lo, t_hi;
+    bool ok = true;
+    int last_it = -1;                                     // latest unit this lane issued a copy for
+    while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi)) {
+        const Problem& pr = P.p[p - 1];
+        const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row);
+        const int T = t_hi - t_lo;
+        const Plan pl = plan_of(G, T, W);
+        // Lane l feeds warp l: its units are l, l + W, ...; (tile, panel) and (stage, phase) move by fixed steps.  The
+        // lanes advance independently: each probes ITS stage (without suspending) and issues its next copy as soon as
+        // its warp has released the stage, so a slow consumer warp never holds back the copies of the others.
+        const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
+        int tj = pl.split ? lane / G.n_panels : lane * pl.tpu;
+        int pn = pl.split ? lane % G.n_panels : 0;
+        int slot = (it0 + lane) % P.slots;
+        int use = (it0 + lane) / P.slots;                      // how often the stage has been used before
+        int s = lane < W ? lane : pl.n_units;                  // this lane's next unit
+        long long t_wait = 0;
+        int spins = 0;
+        while (__any_sync(0xffffffffu, s < pl.n_units)) {
+            if (!waited && __any_sync(0xffffffffu, s < pl.n_units && use > 0)) {
+                // The consumers only start after the previous kernel of the stream has finished; wait for it here
+                // (a wait the stream itself bounds), so that the bounded waits below measure this CTA only.
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                waited = true;
+            }
+            bool progressed = false;
+            if (s < pl.n_units && (use == 0 || mbar_test_wait(smem_u32(&s_empty[slot]), (uint32_t)((use - 1) & 1)))) {
+                const uint32_t bar = smem_u32(&s_full[slot]);
+                const uint32_t dst = smem_u32(ring + (size_t)slot * P.slot_bytes);
+                if (tj >= T) {
+                    mbar_arrive(bar);                           // padding: an empty unit
+                } else if (G.contig) {
+                    // the unit is one run of the plane; rows past the end of the matrix are not fetched
+                    const long long row0 = (long long)(t_lo + tj) * 16;
+                    const long long rows = min((long long)min(pl.tpu, T - tj) * 16, pr.N - row0);
+                    const uint32_t bytes = (uint32_t)rows * (uint32_t)G.row_bytes;
+                    mbar_arrive_expect_tx(bar, bytes);
+                    bulk_g2s(dst, pr.packed + row0 * G.row_bytes, bytes, bar);
+                    last_it = it0 + s;
+                } else {
+                    mbar_arrive_expect_tx(bar, (uint32_t)(16 * G.stride));     // the whole box, zeros included
+                    tensor_g2s(dst, &P.tm[p - 1], pn * G.panel_qc * 8, (t_lo + tj) * 16, bar);
+                    last_it = it0 + s;
+                }
+                if (pl.split) {
+                    tj += step_t; pn += step_p;
+                    if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
+                } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
+                slot += W;
+                if (slot >= P.slots) { slot -= P.slots; ++use; }
+                s += W;
+                progressed = true;
+            }
+            // bounded: no lane made progress for the wait limit
+            if (__any_sync(0xffffffffu, progressed)) { spins = 0; t_wait = 0; }
+            else {
+                __nanosleep(kProducerNapNs);                      // every stage is full: leave the issue slots to the multiplying warps
+                if (++spins >= 64) {
+                    spins = 0;
+                    const long long now = clock64();
+                    if (t_wait == 0) t_wait = now;
+                    const bool give_up = *abort_flag || now - t_wait > P.wait_cycles;
+                    if (__any_sync(0xffffffffu, give_up)) { *abort_flag = 1; ok = false; break; }
+                }
+            }
+        }
+        it0 += pl.n_units;
+    }
+    if (!ok && lane < W) {
+        // gave up: copies already issued still write into this CTA's shared memory; wait for them (bounded).  A lane's
+        // stages are its own, so the phase of a stage's latest use stays complete once its copy has landed.
+        const long long t0 = clock64();
+        for (int it = last_it; it >= 0 && it > last_it - P.slots; it -= W) {
+            const uint32_t bar = smem_u32(&s_full[it % P.slots]);
+            while (!mbar_try_wait(bar, (uint32_t)((it / P.slots) & 1), 1000) && clock64() - t0 < P.wait_cycles) {}
+        }
+    }
+}
+
 template <int NP>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream(const __grid_constant__ Params<NP> P) {
@@ -623,87 +721,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
     }
 
     if (warp == W) {
-        // ------------------------------------------------------------------ producer warp: lane l < W feeds warp l's stages
-        int it0 = 0;                                          // units of the segments before this one (a multiple of W)
-        bool waited = !P.pdl;
-        int p = p_first, t_lo, t_hi;
-        bool ok = true;
-        int last_it = -1;                                     // latest unit this lane issued a copy for
-        while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi)) {
-            const Problem& pr = P.p[p - 1];
-            const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row);
-            const int T = t_hi - t_lo;
-            const Plan pl = plan_of(G, T, W);
-            // Lane l feeds warp l: its units are l, l + W, ...; (tile, panel) and (stage, phase) move by fixed steps.  The
-            // lanes advance independently: each probes ITS stage (without suspending) and issues its next copy as soon as
-            // its warp has released the stage, so a slow consumer warp never holds back the copies of the others.
-            const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
-            int tj = pl.split ? lane / G.n_panels : lane * pl.tpu;
-            int pn = pl.split ? lane % G.n_panels : 0;
-            int slot = (it0 + lane) % P.slots;
-            int use = (it0 + lane) / P.slots;                      // how often the stage has been used before
-            int s = lane < W ? lane : pl.n_units;                  // this lane's next unit
-            long long t_wait = 0;
-            int spins = 0;
-            while (__any_sync(0xffffffffu, s < pl.n_units)) {
-                if (!waited && __any_sync(0xffffffffu, s < pl.n_units && use > 0)) {
-                    // The consumers only start after the previous kernel of the stream has finished; wait for it here
-                    // (a wait the stream itself bounds), so that the bounded waits below measure this CTA only.
-                    asm volatile("griddepcontrol.wait;" ::: "memory");
-                    waited = true;
-                }
-                bool progressed = false;
-                if (s < pl.n_units && (use == 0 || mbar_test_wait(smem_u32(&s_empty[slot]), (uint32_t)((use - 1) & 1)))) {
-                    const uint32_t bar = smem_u32(&s_full[slot]);
-                    const uint32_t dst = smem_u32(ring + (size_t)slot * P.slot_bytes);
-                    if (tj >= T) {
-                        mbar_arrive(bar);                           // padding: an empty unit
-                    } else if (G.contig) {
-                        // the unit is one run of the plane; rows past the end of the matrix are not fetched
-                        const long long row0 = (long long)(t_lo + tj) * 16;
-                        const long long rows = min((long long)min(pl.tpu, T - tj) * 16, pr.N - row0);
-                        const uint32_t bytes = (uint32_t)rows * (uint32_t)G.row_bytes;
-                        mbar_arrive_expect_tx(bar, bytes);
-                        bulk_g2s(dst, pr.packed + row0 * G.row_bytes, bytes, bar);
-                        last_it = it0 + s;
-                    } else {
-                        mbar_arrive_expect_tx(bar, (uint32_t)(16 * G.stride));     // the whole box, zeros included
-                        tensor_g2s(dst, &P.tm[p - 1], pn * G.panel_qc * 8, (t_lo + tj) * 16, bar);
-                        last_it = it0 + s;
-                    }
-                    if (pl.split) {
-                        tj += step_t; pn += step_p;
-                        if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
-                    } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
-                    slot += W;
-                    if (slot >= P.slots) { slot -= P.slots; ++use; }
-                    s += W;
-                    progressed = true;
-                }
-                // bounded: no lane made progress for the wait limit
-                if (__any_sync(0xffffffffu, progressed)) { spins = 0; t_wait = 0; }
-                else {
-                    __nanosleep(kProducerNapNs);                      // every stage is full: leave the issue slots to the multiplying warps
-                    if (++spins >= 64) {
-                        spins = 0;
-                        const long long now = clock64();
-                        if (t_wait == 0) t_wait = now;
-                        const bool give_up = *abort_flag || now - t_wait > P.wait_cycles;
-                        if (__any_sync(0xffffffffu, give_up)) { *abort_flag = 1; ok = false; break; }
-                    }
-                }
-            }
-            it0 += pl.n_units;
-        }
-        if (!ok && lane < W) {
-            // gave up: copies already issued still write into this CTA's shared memory; wait for them (bounded).  A lane's
-            // stages are its own, so the phase of a stage's latest use stays complete once its copy has landed.
-            const long long t0 = clock64();
-            for (int it = last_it; it >= 0 && it > last_it - P.slots; it -= W) {
-                const uint32_t bar = smem_u32(&s_full[it % P.slots]);
-                while (!mbar_try_wait(bar, (uint32_t)((it / P.slots) & 1), 1000) && clock64() - t0 < P.wait_cycles) {}
-            }
-        }
+        producer_warp(P, lo, hi, p_first, W, ring, s_full, s_empty, abort_flag, lane);
     } else {
         // ------------------------------------------------------------------ consumer warps
         const int g = lane >> 2, t = lane & 3;
@@ -939,6 +957,7 @@ struct HostProblem {
     const uint16_t* ovf_col;
     const void* x;
     float* y;
+    int64_t B;
 };
 
 inline size_t xs_bytes_of(const Geo& g, int r) { return (size_t)g.n_qc * ((128 / r) / 16) * 256; }
@@ -998,7 +1017,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         q.packed = hp[i].packed; q.alpha = hp[i].alpha; q.zero = hp[i].zero;
         q.ovf_row_ptr = hp[i].ovf_row_ptr; q.ovf_col = hp[i].ovf_col;
         q.x = static_cast<const __nv_bfloat16*>(hp[i].x); q.y = hp[i].y;
-        q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.pad_ = 0;
+        q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.B = 1;
         q.item0 = item0;
         const Geo g = geometry(q.N, q.K, q.r, unit_row);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;

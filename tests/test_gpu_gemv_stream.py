@@ -149,7 +149,8 @@ def test_grouped_mixed_list():
 def test_grouped_long_list_and_equality_with_single_calls():
     # more problems than the small descriptor table holds; every output must equal, bit for bit, what matq_gemv's
     # persistent path gives for the problem alone (integer sums do not depend on how the list is cut)
-    shapes = [(300 + 37 * i, 128 * (1 + i % 9), (8, 4, 2)[i % 3]) for i in range(21)]
+    # (the long rows change the number of multiplying warps of the launch: the fp32 sum of x must not depend on it)
+    shapes = [(300 + 37 * i, 128 * (1 + i % 9), (8, 4, 2)[i % 3]) for i in range(21)] + [(130, 9216, 4), (77, 14336, 2)]
     hosts = [_problem(N, K, r, 50 + i) for i, (N, K, r) in enumerate(shapes)]
     devs = [_to_device(p) for p in hosts]
     mq.gemv_grouped(devs)
