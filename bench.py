@@ -238,14 +238,14 @@ class DeviceStack:
             self.x8[i].view(torch.uint16).copy_(torch.from_numpy(x))
         torch.cuda.synchronize()
 
-    def problems(self, nm, r, ep, idx):
-        """matq_gemv_grouped descriptors (B = 1) of the matrices `idx`."""
-        key = (nm, r, ep, tuple(idx))
+    def problems(self, nm, r, ep, idx, batch=False):
+        """matq_gemv_grouped descriptors of the matrices `idx`: the first activation vector, or all eight (`batch`)."""
+        key = (nm, r, ep, tuple(idx), batch)
         if key not in self._groups:
             planes = self.p4 if r == 4 else self.p2
             self._groups[key] = self.mq.gemv_group([
                 dict(packed=planes[i], K=self.shapes[i][4], r=r, alpha=self.alpha[i], zero=self.zero[i],
-                     x=self.x8[i][0], y=self.y[nm][i][0],
+                     x=self.x8[i] if batch else self.x8[i][0], y=self.y[nm][i] if batch else self.y[nm][i][0],
                      ovf_row_ptr=self.rp[i] if ep else None, ovf_col=self.col[i] if ep else None) for i in idx])
         return self._groups[key]
 
@@ -268,6 +268,16 @@ class DeviceStack:
                 mq.gemv_grouped(g, flags=mq.GEMV_PDL, dev_status=self.status)
         return run, sum((len(g) + 127) // 128 for g in groups)
 
+    def gemv_b8_per_matrix(self, nm, r):
+        """B = 8 with one matq_gemv (the bf16 tensor kernel) per matrix: the comparison for the whole-stack call."""
+        mq, n, S = self.mq, len(self.shapes), self.shapes
+        planes = self.p4 if r == 4 else self.p2
+
+        def run():
+            for i in range(n):
+                mq.gemv(planes[i], S[i][4], r, self.alpha[i], self.zero[i], self.x8[i], y=self.y[nm][i], flags=mq.GEMV_AUTO | mq.GEMV_PDL)
+        return run, n
+
     # stage-major plan: (name, callable over the whole stack, kernels launched, algorithmic bytes)
     def stages(self):
         mq = self.mq
@@ -288,13 +298,12 @@ class DeviceStack:
                               ovf_col=self.col[i], ovf_capacity=self.cap[i], ovf_count=self.cnt[i], dev_status=self.status)
 
         def gemv_b8(nm, r):
-            planes = self.p4 if r == 4 else self.p2
+            """B = 8 over the whole stack in one matq_gemv_grouped call."""
+            g = self.problems(nm, r, False, list(range(n)), batch=True)
 
             def run():
-                for i in range(n):
-                    mq.gemv(planes[i], S[i][4], r, self.alpha[i], self.zero[i], self.x8[i], y=self.y[nm][i],
-                            flags=mq.GEMV_AUTO | mq.GEMV_PDL)
-            return run
+                mq.gemv_grouped(g, flags=mq.GEMV_PDL, dev_status=self.status)
+            return run, mq.gemv_grouped_launches(g)
 
         nnz = getattr(self, "nnz", [0] * n)
         g4, l4 = self.gemv_b1("g4b1", 4, False, n)
@@ -306,8 +315,8 @@ class DeviceStack:
             ("slice_pack_r2_ep", sp2, 2 * n, sum(bytes_slice_pack(N, K, 2, z) for (_, _, _, N, K), z in zip(S, nnz))),
             # the decode stages come last, the B = 1 ones after the B = 8 ones: a stage that directly follows slice_pack
             # also pays the write-back of the planes that stage left dirty in the L2, which no decode loop ever sees
-            ("gemv_r4_b8", gemv_b8("g4b8", 4), n, sum(bytes_gemv(N, K, 4, 8) for (_, _, _, N, K) in S)),
-            ("gemv_r2_b8", gemv_b8("g2b8", 2), n, sum(bytes_gemv(N, K, 2, 8) for (_, _, _, N, K) in S)),
+            ("gemv_r4_b8", *gemv_b8("g4b8", 4), sum(bytes_gemv(N, K, 4, 8) for (_, _, _, N, K) in S)),
+            ("gemv_r2_b8", *gemv_b8("g2b8", 2), sum(bytes_gemv(N, K, 2, 8) for (_, _, _, N, K) in S)),
             ("gemv_r4_b1", g4, l4, sum(bytes_gemv(N, K, 4, 1) for (_, _, _, N, K) in S)),
             ("gemv_r2_b1", g2, l2, sum(bytes_gemv(N, K, 2, 1) for (_, _, _, N, K) in S)),
             ("gemv_r2_ep_b1", gep, lep, sum(bytes_gemv(N, K, 2, 1, z) for (_, _, _, N, K), z in zip(S, nnz))),
@@ -439,8 +448,12 @@ def run_cuda(args, rank, world, local_rank):
             ms = time_graph(torch, capture(torch, fn))
             stages[f"{key}_{label}"] = dict(gemv_entry(ms, nbytes, peaks, launches), in_step=False)
             gemv_frac[f"cfg2_{key[5:]}_{label}"] = stages[f"{key}_{label}"]["frac_hbm"]
-    gemv_frac["cfg2_r4_b8_launch_per_matrix"] = stages["gemv_r4_b8"]["frac_hbm"]
-    gemv_frac["cfg2_r2_b8_launch_per_matrix"] = stages["gemv_r2_b8"]["frac_hbm"]
+    for nm, r, key in (("g4b8", 4, "gemv_r4_b8"), ("g2b8", 2, "gemv_r2_b8")):
+        gemv_frac[f"cfg2_{key[5:]}_whole_stack_call"] = stages[key]["frac_hbm"]
+        fn, launches = st.gemv_b8_per_matrix(nm, r)
+        ms = time_graph(torch, capture(torch, fn))
+        stages[f"{key}_launch_per_matrix"] = dict(gemv_entry(ms, plan[names.index(key)][3], peaks, launches), in_step=False)
+        gemv_frac[f"cfg2_{key[5:]}_launch_per_matrix"] = stages[f"{key}_launch_per_matrix"]["frac_hbm"]
 
     gpu_launches = sum(p[2] for p in plan)
 
@@ -487,8 +500,8 @@ def run_cuda(args, rank, world, local_rank):
             "data": "synthetic",
             "config": {"workload": f"configs[1] Gemma-2-2B-shaped MLP decode stack, {args.layers} layers x (gate,up 9216x2304; down 2304x9216), "
                                    "bf16 N(0,0.02) weights, x bf16 N(0,1)",
-                       "step": "quantize -> slice_pack r=4 -> slice_pack r=2 + extra-precision lists -> gemv r=4, r=2 at B=8 (launch per matrix) "
-                               "-> gemv r=4, r=2, r=2 E.P. at B=1 (matq_gemv_grouped, whole stack per call)"
+                       "step": "quantize -> slice_pack r=4 -> slice_pack r=2 + extra-precision lists -> gemv r=4, r=2 at B=8 -> gemv r=4, r=2, r=2 E.P. at B=1 "
+                               "(all decode stages: matq_gemv_grouped, whole stack per call)"
                                "; dense multi-precision forward measured separately (gemm_multi_cfg4)",
                        "value_definition": "decode GEMV at B = 1: algorithmic HBM bytes of the gemv_r4_b1 and gemv_r2_b1 stages / their device time "
                                            f"({round(gemv_ms, 4)} ms of the step); step_GBps is the same ratio over all stages",
@@ -573,6 +586,14 @@ def _gemv_cases(mq, torch, shapes, planes, r, xs, ys, al, Bs, per_layer, peaks, 
         out[f"r{r}_b{B}_launch_per_matrix"] = gemv_entry(ms, nbytes, peaks, n)
         gemv_frac[f"{prefix}_r{r}_b{B}_launch_per_matrix"] = out[f"r{r}_b{B}_launch_per_matrix"]["frac_hbm"]
         if B != 1:
+            if ep:
+                continue
+            # batches: the whole stack in one matq_gemv_grouped call (the batched persistent kernel)
+            g = mq.gemv_group([dict(packed=planes[i], K=K, r=r, alpha=al[i], zero=al[i], x=xs[i][:B], y=ys[i][:B])
+                               for i, (N, K) in enumerate(shapes)])
+            ms = time_graph(torch, capture(torch, lambda: mq.gemv_grouped(g, flags=mq.GEMV_PDL)), reps=5)
+            out[f"r{r}_b{B}_whole_stack_call"] = gemv_entry(ms, nbytes, peaks, mq.gemv_grouped_launches(g))
+            gemv_frac[f"{prefix}_r{r}_b{B}_whole_stack_call"] = out[f"r{r}_b{B}_whole_stack_call"]["frac_hbm"]
             continue
         probs = [dict(packed=planes[i], K=K, r=r, alpha=al[i], zero=al[i], x=xs[i][0], y=ys[i][0],
                       ovf_row_ptr=rps[i] if ep else None, ovf_col=cols[i] if ep else None) for i, (N, K) in enumerate(shapes)]
@@ -597,7 +618,8 @@ def gemv_cfg3(mq, torch, peaks, gemv_frac):
     shapes = [s for _ in range(layers) for s in per_layer]
     out = {"workload": f"configs[2] Gemma-2-9B decoder stack, {layers} layers x (q, k, v, o, gate, up, down), r = 8, 4, 2 at B = 1, 4, 16; "
                        "B = 1: one launch per matrix (PDL chain), one matq_gemv_grouped call per layer, one for the whole stack; "
-                       "B = 4, 16: one launch per matrix; one CUDA graph per case"}
+                       "B = 4, 16: one launch per matrix (bf16 tensor kernel) and one matq_gemv_grouped call for the whole stack (batched "
+                       "integer kernel); one CUDA graph per case"}
     xs = [torch.randn(16, k, device="cuda").to(torch.bfloat16) for n, k in shapes]
     ys = [torch.empty(16, n, device="cuda") for n, k in shapes]
     al = [torch.ones(n, device="cuda") for n, k in shapes]

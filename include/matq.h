@@ -222,6 +222,8 @@ typedef struct matq_gemv_problem {
 } matq_gemv_problem;
 int matq_gemv_grouped(const matq_gemv_problem *problems, int n_problems, int c, unsigned flags,
                       int32_t *dev_status, void *stream);
+/* Number of kernel launches matq_gemv_grouped makes for this list (host only, launches nothing); -1 for a list it would refuse. */
+int matq_gemv_grouped_launches(const matq_gemv_problem *problems, int n_problems);
 
 /*
  * (4) Multi-precision dense forward of MatQuant co-training (Eq. 7): for every

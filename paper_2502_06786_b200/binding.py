@@ -24,7 +24,7 @@ GEMV_TEST_STALL = 0x8000
 TEACHER_AND_TARGET = 256    # matq_gemm_multi_loss: teacher[i] = TEACHER_AND_TARGET + j
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
-           "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped",
+           "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped", "matq_gemv_grouped_launches",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
            "matq_gemm_multi_loss_workspace_bytes", "matq_gemm_multi_loss",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
@@ -67,6 +67,8 @@ def _load():
     lib.matq_gemv.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp, i32, i64, vp, i64, vp, sz, u32, vp, vp]
     lib.matq_gemv_grouped.restype = i32
     lib.matq_gemv_grouped.argtypes = [C.POINTER(GemvProblem), i32, i32, u32, vp, vp]
+    lib.matq_gemv_grouped_launches.restype = i32
+    lib.matq_gemv_grouped_launches.argtypes = [C.POINTER(GemvProblem), i32]
     lib.matq_gemm_multi_workspace_bytes.restype = sz
     lib.matq_gemm_multi_workspace_bytes.argtypes = [i32, i64, i64, i64, i32]
     lib.matq_gemm_multi.restype = i32
@@ -250,6 +252,13 @@ def gemv_grouped(group, flags=0, dev_status=None, c=8, raise_on_error=True):
     st = _lib.matq_gemv_grouped(group, len(group), c, int(flags), _ptr(dev_status), _stream())
     _check(st, "matq_gemv_grouped", raise_on_error)
     return st
+
+
+def gemv_grouped_launches(group) -> int:
+    """Kernel launches gemv_grouped makes for this descriptor array."""
+    if not isinstance(group, C.Array):
+        group = gemv_group(group)
+    return int(_lib.matq_gemv_grouped_launches(group, len(group)))
 
 
 def gemm_multi_workspace_bytes(src_kind, M, N, K, n_r) -> int:

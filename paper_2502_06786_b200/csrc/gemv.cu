@@ -73,6 +73,32 @@ extern "C" int matq_gemv_grouped(const matq_gemv_problem* problems, int n_proble
     return gstream::launch_batch(many.data(), many_b.data(), (int)many.size(), pdl, wait, stall, dev_status, s);
 }
 
+extern "C" int matq_gemv_grouped_launches(const matq_gemv_problem* problems, int n_problems) {
+    using namespace matq;
+    if (n_problems < 0 || (n_problems > 0 && !problems)) return -1;
+    const gstream::HostProblem* hp = reinterpret_cast<const gstream::HostProblem*>(problems);
+    std::vector<gstream::HostProblem> one, many;
+    std::vector<int> many_b;
+    for (int i = 0; i < n_problems; ++i) {
+        if (hp[i].N == 0) continue;
+        if (hp[i].B <= 1) { one.push_back(hp[i]); continue; }
+        if (gstream::split_batch(hp[i], one, many, many_b) != MATQ_OK) return -1;
+    }
+    int launches = 0;
+    const size_t per = one.size() <= (size_t)gstream::kSmallList ? gstream::kSmallList : gstream::kLargeList;
+    for (size_t i = 0; i < one.size(); i += per) {
+        bool lists = false;
+        for (size_t j = i; j < std::min(one.size(), i + per); ++j) lists = lists || one[j].ovf_row_ptr != nullptr;
+        launches += lists ? 2 : 1;                                  // ep_rowsum + the persistent kernel
+    }
+    for (int G = 1; G <= 4; G *= 2) {
+        size_t cnt = 0;
+        for (int b : many_b) cnt += gstream::groups_of(b) == G;
+        launches += (int)((cnt + gstream::kLargeList - 1) / gstream::kLargeList);
+    }
+    return launches;
+}
+
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {
     (void)N; (void)K; (void)r; (void)B;
     return 0;   // the K-split is reduced inside warps / CTAs; no scratch is needed
