@@ -177,6 +177,8 @@ int matq_slice_pack(const uint8_t *q, int64_t N, int64_t K, int c, int r, int ex
  *   products of the fields with the activations scaled to 30-bit integers by a power of two taken from
  *   max |x| (an activation below 2^-22 of the largest is rounded to an absolute 2^-24 of the largest at worst),
  *   then applies alpha and z in fp32; other batches accumulate bf16 x bf16 products in fp32.
+ *   MATQ_GEMV_STREAM with B > 1 (dense rows: ldx == K, ldy == N; no lists) takes the batched integer kernel
+ *   described under (3b).
  */
 size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B);
 int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
@@ -187,22 +189,33 @@ int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
               int32_t *dev_status, void *stream);
 
 /*
- * (3b) Several decode GEMVs (B = 1) in ONE launch.  A decoder layer multiplies the same activation vector with
+ * (3b) Several decode GEMVs in ONE launch.  A decoder layer multiplies the same activation vector with
  *      several weight matrices (the query, key and value projections; the gate and up projections of the FFN,
  *      Sections 1 and 5.3), a Mix'n'Match model (Section 3.2.1, Appendix B) gives every layer its own r, and each
  *      plane is only a few megabytes, i.e. a few microseconds of HBM time: a launch per plane is bound by launch
  *      latency, not by the weight traffic that Section 1 names as the cost of decoding.  This call takes a list of
- *      independent problems, each exactly a matq_gemv with B = 1,
- *        y_i[n] = sum_k x_i[k] * alpha_i[n] * (S_i[n,k] - z_i[n])        (+ Eq. 8's extra bucket where a list is given),
- *      and runs them with one persistent kernel whose CTAs share the list's bytes evenly, whatever the shapes.
- *      Problems may share x or not, may differ in N, K and r, and must not depend on one another (no y_i may be
- *      an x_j of the same call).  Results are those of matq_gemv's integer path (exact integer sums, reproducible,
- *      independent of how the list is split over CTAs).
+ *      independent problems, each a matq_gemv,
+ *        y_i[b,n] = sum_k x_i[b,k] * alpha_i[n] * (S_i[n,k] - z_i[n])    (+ Eq. 8's extra bucket where a list is given),
+ *      and runs them with persistent kernels whose CTAs share the list's bytes evenly, whatever the shapes.
+ *      Problems may share x or not, may differ in N, K, r and B, and must not depend on one another (no y_i may be
+ *      an x_j of the same call).  With one vector per problem (B <= 1) the results are those of matq_gemv's integer
+ *      path (exact integer sums, reproducible: a problem gives the same bits alone, in any list and however the list
+ *      is split over CTAs).
+ *      Batches (2 <= B <= 16, no lists): the plane is read from HBM once for up to 8 vectors.  The sums are exact
+ *      integers again, but an activation is a 22-bit integer relative to the largest magnitude of ITS vector, and a
+ *      field that sits s bits up in its byte meets its activation divided by 2^s: the rounding step is 2^-22 (r = 8),
+ *      2^-18 (r = 4), 2^-16 (r = 2) of twice the vector's largest magnitude (about 1e-6, 2e-5, 6e-5 of rms(y) for
+ *      Gaussian activations).  A vector whose largest element is thousands of times its typical one loses
+ *      accordingly; such vectors belong in problems of their own (B = 1: 30-bit activations) or in matq_gemv's
+ *      default path (bf16 products).  A batch that does not fit one launch's shared memory (more than 8 vectors;
+ *      more than 4 at K = 9216) is cut into problems that share the plane; r = 2 batches need K % 256 == 0.
  *   problems   in   HOST array of n_problems descriptors; the pointers inside are DEVICE pointers:
  *                     packed uint8 [N, K*r/8] 16-byte aligned, alpha / zero fp32 [N], ovf_row_ptr / ovf_col both NULL
- *                     or both given, x bf16 [K] 16-byte aligned, y fp32 [N].  r in {8, 4, 2}, K % 128 == 0, K <= 32768.
+ *                     or both given (B <= 1 only), x bf16 [K] (or [B, K], rows K apart) 16-byte aligned, y fp32 [N]
+ *                     (or [B, N], rows N apart).  r in {8, 4, 2}, K % 128 == 0, K <= 32768.
  *                     A problem with N == 0 is skipped.  The array is read during the call only.
- *   n_problems      any number >= 0; up to 128 problems share a launch, longer lists take several
+ *   n_problems      any number >= 0; up to 128 problems share a launch, longer lists take several; single vectors
+ *                   and batches of 2, 3-4 and 5-8 vectors go to launches of their own
  *   flags           0 or MATQ_GEMV_PDL (MATQ_GEMV_TEST_STALL for tests of the error path; meaning of PDL as for matq_gemv: no plane, alpha, zero or list of the call is
  *                   written by the previous kernel of the stream)
  *   A wait inside the kernel that does not end within about two seconds sets dev_status = MATQ_ERR_TIMEOUT; the
