@@ -176,12 +176,13 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // ---------------- epilogue: thread = one output row (TMEM lane), 32 columns at a time
         const int quad = warp & 3;
         const int64_t m = m0 + quad * 32 + lane;
-        const bool done = mbar_wait(smem_u32(&s_acc), 0);
+        // whole warps agree on the outcome: the reads of tensor memory below are warp-wide
+        const bool done = __all_sync(0xffffffffu, mbar_wait(smem_u32(&s_acc), 0));
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (!done) s_timeout = 1;
+        if (!done) s_timeout = 1;                           // gave up: report it, read and store nothing
         const float sx = (m < P.M) ? P.sx[m] : 0.f;
         float lacc[kMaxR] = {0.f, 0.f, 0.f};               // loss mode: this thread's squared errors per precision
-        for (int r = 0; r < P.n_r; ++r) {
+        for (int r = 0; r < (done ? P.n_r : 0); ++r) {
             const int pr = P.wide ? 0 : r;                    // which precision this accumulator belongs to
             const int64_t nb = n0 + (P.wide ? r * kBN : 0);     // first channel of this accumulator
             const float* al = s_alpha + (P.wide ? r * kBN : 0);

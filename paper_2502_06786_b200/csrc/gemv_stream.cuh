@@ -111,7 +111,8 @@ struct Params {
     int slot_bytes;
     int xs_bytes;             // staged activation bytes (largest problem)
     int W;                    // consumer warps
-    int pdl;
+    int pdl;                  // 0: plain launch; 1: programmatic dependent of an unknown kernel (wait before x is read);
+                              // 2: dependent of ep_rowsum, released after that kernel's own wait (wait before its sums are read)
     int unit_row;             // bytes per row of the largest unit
     int hold;                 // diagnostics: the producer issues no copies, so every wait for a stage runs out
 };
@@ -524,10 +525,11 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(ep_smem);      // the problem's activations
     const int tid = threadIdx.x, sub = tid & 7, grp = tid >> 3;          // eight lanes per row, 2 x 64 rows per pass
     const unsigned gmask = 0xffu << (tid & 24);
-    if (P.pdl) {
-        asm volatile("griddepcontrol.launch_dependents;");
-        asm volatile("griddepcontrol.wait;" ::: "memory");               // x may be written by the previous kernel
-    }
+    // x may be written by the previous kernel.  The persistent kernel behind this one is released only after that
+    // wait: once it runs, x is final, so it may stage x and multiply while these sums are still being taken, and it
+    // waits for this kernel only before it reads the first sum.
+    if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
     const long long lo = P.rows * blockIdx.x / gridDim.x, hi = P.rows * (blockIdx.x + 1) / gridDim.x;
     for (int p = 0; p < P.n; ++p) {
         const EpProblem& pr = P.p[p];
@@ -598,7 +600,7 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
                                               uint64_t* s_full, uint64_t* s_empty, volatile int* abort_flag, int lane) {
     // ------------------------------------------------------------------ producer warp: lane l < W feeds warp l's stages
     int it0 = 0;                                          // units of the segments before this one (a multiple of W)
-    bool waited = !P.pdl;
+    bool waited = P.pdl != 1;
     int p = p_first, t_lo, t_hi;
     bool ok = true;
     int last_it = -1;                                     // latest unit this lane issued a copy for
@@ -730,6 +732,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         int split_tiles = 0;                                   // split-mode tiles of earlier segments (a tile's slot = its count mod kTileSlots)
         int p = p_first, t_lo, t_hi;
         bool first = true;
+        bool ep_ready = P.pdl != 2;                            // whether ep_rowsum's sums may be read yet
         Geo G;
         float xsum = 0.f;
         int xexp = 0;
@@ -754,7 +757,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 // wait; pulling their lines into the L2 earlier is harmless (the L2 is the point of coherence) and takes the
                 // HBM latency of a cold vector off the critical path.
                 for (int i = ctid * 64; i < pr.K; i += nthr * 64) asm volatile("prefetch.global.L2 [%0];" ::"l"(pr.x + i));
-                if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+                if (P.pdl == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
             }
             first = false;
 
@@ -826,20 +829,29 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             float sc[kMaxTpu], sc_next[kMaxTpu];
             float epv[kMaxTpu], epv_next[kMaxTpu];                    // extra precision: the sparse term of a tile's rows (lanes 0-15)
             const bool ep = pr.ovf_row_ptr != nullptr;
-            // the sparse term was left in y by ep_rowsum, which this kernel has waited for (plain coherent loads)
+            // The sparse term is left in y by ep_rowsum (plain coherent loads).  Behind that kernel (pdl == 2) this one
+            // starts before the sums are complete: it waits for them when it first needs one, and until then the loads a
+            // round ahead are skipped (`epv_ok` / `epv_next_ok`: whether the registers hold loaded values).
             auto load_ep = [&](long long row0) -> float {
                 const long long row = row0 + lane;
                 float v = 0.f;
                 if (lane < 16 && row < pr.N) asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(pr.y + row) : "memory");
                 return v;
             };
+            bool epv_ok = false, epv_next_ok = ep_ready;
 #pragma unroll
             for (int k = 0; k < kMaxTpu; ++k) {
                 sc[k] = 0.f; sc_next[k] = sc_first[k];                      // tile mode: the first unit's tiles
                 epv[k] = 0.f;
                 const int tn = warp * pl.tpu + k;
-                epv_next[k] = (ep && !pl.split && k < pl.tpu && tn < T) ? load_ep((long long)(t_lo + tn) * 16) : 0.f;
+                epv_next[k] = (ep && ep_ready && !pl.split && k < pl.tpu && tn < T) ? load_ep((long long)(t_lo + tn) * 16) : 0.f;
             }
+            auto await_ep = [&]() {
+                if (!ep_ready) {
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    ep_ready = true;
+                }
+            };
             // split mode: the partial sums of tile `cur` go to its accumulator in shared memory; the warp that brings the
             // last of a tile's contributions finishes it (returns true for that warp, with the sums in acc[0])
             auto flush = [&]() -> bool {
@@ -879,6 +891,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             uint32_t parity = (uint32_t)(((it0 + warp) / P.slots) & 1);
             // split mode: the warp that completes a tile finishes it
             auto finish_split = [&](long long row0, float scales) {
+                if (ep) await_ep();
                 const float ep_rows = ep ? load_ep(row0) : 0.f;
                 finish_tile(pr.y, pr.N, sh, xexp, xsum, row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], scales, ep_rows, lane, !*abort_flag);
             };
@@ -899,9 +912,11 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                         const int tn = tj + W * pl.tpu + k;                  // the same warp's next group of tiles, a round ahead
                         if (k < pl.tpu && tn < T) {
                             sc_next[k] = load_scales((long long)(t_lo + tn) * 16);
-                            if (ep) epv_next[k] = load_ep((long long)(t_lo + tn) * 16);
+                            if (ep && ep_ready) epv_next[k] = load_ep((long long)(t_lo + tn) * 16);
                         }
                     }
+                    epv_ok = epv_next_ok;
+                    epv_next_ok = ep_ready;
                     zero_acc(acc);
                 }
                 const bool landed = wait_phase(smem_u32(&s_full[slot]), parity, abort_flag, P.wait_cycles);
@@ -916,6 +931,13 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     }
                     if (tile_done) {
                         fold(acc);
+                        if (ep && !epv_ok) {                                  // not loaded a round ahead: wait for the sums, load them now
+                            await_ep();
+#pragma unroll
+                            for (int kk = 0; kk < kMaxTpu; ++kk)
+                                if (kk < n_tiles) epv[kk] = load_ep((long long)(t_lo + tj + kk) * 16);
+                            epv_ok = true;
+                        }
                         finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
                                     k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3],
                                     k == 0 ? epv[0] : k == 1 ? epv[1] : k == 2 ? epv[2] : epv[3], lane, !*abort_flag);
@@ -1035,6 +1057,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     // flight matter more than the eighth warp.
     if (W == kMaxW && fit / (W - 1) * (W - 1) > fit / W * W) --W;
     const int slots = fit / W * W;
+    bool behind_ep = false;
     // Extra precision: the sparse term of every problem with lists goes to its y first (see ep_rowsum); the persistent
     // kernel then runs as that kernel's programmatic dependent (it touches y only after its dependency wait).
     {
@@ -1066,10 +1089,11 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
             ec.numAttrs = pdl ? 1 : 0;
             if (cudaLaunchKernelEx(&ec, ek, E) != cudaSuccess) { cudaGetLastError(); return MATQ_ERR_CUDA; }
             pdl = true;
+            behind_ep = true;
         }
     }
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
-    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
     auto kern = gemv_stream<NP>;
     if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};

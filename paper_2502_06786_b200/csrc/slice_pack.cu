@@ -189,45 +189,24 @@ ovf_scan(int32_t* __restrict__ row_ptr, int64_t N, int64_t capacity, int64_t* __
     }
 }
 
-// One warp per row writes the ascending column indices of the overflow elements.
-template <bool VEC>
+// One warp per row writes the ascending column indices of the overflow elements, one code per lane and step (rows
+// whose length or alignment the vectorised variant below does not take).
 __global__ void __launch_bounds__(kSliceThreads)
 ovf_fill(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, const int32_t* __restrict__ row_ptr,
          const int64_t* __restrict__ total, int64_t capacity, uint16_t* __restrict__ ovf_col) {
-    if (*total > capacity || *total > 0x7fffffff) return;   // lists are unspecified in that case
+    if (*total > capacity || *total > 0x7fffffff) return;   // lists are unspecified in that case (ovf_scan has reported it)
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (kSliceThreads / 32);
-    constexpr int kPerLane = VEC ? 16 : 1;
     for (int64_t n = (int64_t)blockIdx.x * (kSliceThreads / 32) + (threadIdx.x >> 5); n < N; n += warps) {
         int64_t out = row_ptr[n];
         if (row_ptr[n + 1] == out) continue;
         const uint8_t* row = q + n * K;
-        for (int64_t k0 = 0; k0 < K; k0 += 32 * kPerLane) {
-            const int64_t k = k0 + (int64_t)lane * kPerLane;
-            uint32_t mask = 0;
-            if (k < K) {
-                if (VEC) {
-                    const uint4 v = ld_stream_u4(row + k);
-                    mask = gather_byte_lsbs(slice4(v.x, r).ov) | (gather_byte_lsbs(slice4(v.y, r).ov) << 4) |
-                           (gather_byte_lsbs(slice4(v.z, r).ov) << 8) | (gather_byte_lsbs(slice4(v.w, r).ov) << 12);
-                } else {
-                    mask = slice4(row[k], r).ov & 1u;
-                }
-            }
-            const int cnt = __popc(mask);
-            int incl = cnt;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            int64_t pos = out + incl - cnt;
-            while (mask) {
-                const int b = __ffs(mask) - 1;
-                ovf_col[pos++] = (uint16_t)(k + b);
-                mask &= mask - 1;
-            }
-            out += __shfl_sync(0xffffffffu, incl, 31);
+        for (int64_t k0 = 0; k0 < K; k0 += 32) {
+            const int64_t k = k0 + lane;
+            const uint32_t mask = k < K ? (slice4(row[k], r).ov & 1u) : 0u;
+            const unsigned ballot = __ballot_sync(0xffffffffu, mask != 0);
+            if (mask) ovf_col[out + __popc(ballot & ((1u << lane) - 1u))] = (uint16_t)k;
+            out += __popc(ballot);
         }
     }
 }
@@ -652,8 +631,7 @@ extern "C" int matq_slice_pack(const uint8_t* q, int64_t N, int64_t K, int c, in
         const int64_t cap = (int64_t)sm_count() * 32;
         if (blocks > cap) blocks = cap;
         if (vec) ovf_fill_batched<<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
-        else if (vec) ovf_fill<true><<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
-        else ovf_fill<false><<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
+        else ovf_fill<<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
     }
     return launch_status();
 }
