@@ -91,12 +91,7 @@ extern "C" int matq_gemv_grouped_launches(const matq_gemv_problem* problems, int
         for (size_t j = i; j < std::min(one.size(), i + per); ++j) lists = lists || one[j].ovf_row_ptr != nullptr;
         launches += lists ? 2 : 1;                                  // ep_rowsum + the persistent kernel
     }
-    for (int G = 1; G <= 4; G *= 2) {
-        size_t cnt = 0;
-        for (int b : many_b) cnt += gstream::groups_of(b) == G;
-        launches += (int)((cnt + gstream::kLargeList - 1) / gstream::kLargeList);
-    }
-    return launches;
+    return launches + gstream::count_batch_launches(many.data(), many_b.data(), (int)many.size());
 }
 
 extern "C" size_t matq_gemv_workspace_bytes(int64_t N, int64_t K, int r, int B) {

@@ -591,20 +591,46 @@ inline int max_groups(int64_t N, int64_t K, int r) {
 inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     for (int i = 0; i < n; ++i)
         if (hp[i].N != 0 && !eligible_batch(hp[i].N, hp[i].K, hp[i].r, hb[i])) return MATQ_ERR_SHAPE;      // before anything is launched
+    // Problems with the same number of groups share a launch, except that those whose staged activations would leave
+    // the launch fewer than seven multiplying warps (long rows) get a launch of their own: the number of warps is a
+    // property of the launch, and the short rows of a stack should not run with four.
     std::vector<HostProblem> sel;
     std::vector<int> sel_b;
-    for (int G = 1; G <= 4; G *= 2) {
-        sel.clear(); sel_b.clear();
-        for (int i = 0; i < n; ++i)
-            if (groups_of(hb[i]) == G) { sel.push_back(hp[i]); sel_b.push_back(hb[i]); }
-        for (size_t i = 0; i < sel.size(); i += kLargeList) {
-            const int cnt = (int)std::min<size_t>(kLargeList, sel.size() - i);
-            const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s)
-                                             : launch_list_batch_g<kLargeList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s);
-            if (st != MATQ_OK) return st;
+    for (int G = 1; G <= 4; G *= 2)
+        for (int wide = 0; wide < 2; ++wide) {
+            sel.clear(); sel_b.clear();
+            for (int i = 0; i < n; ++i) {
+                if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
+                const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
+                const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
+                if ((fit >= kMaxW - 1) != (wide == 0)) continue;
+                sel.push_back(hp[i]); sel_b.push_back(hb[i]);
+            }
+            for (size_t i = 0; i < sel.size(); i += kLargeList) {
+                const int cnt = (int)std::min<size_t>(kLargeList, sel.size() - i);
+                const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s)
+                                                 : launch_list_batch_g<kLargeList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s);
+                if (st != MATQ_OK) return st;
+            }
         }
-    }
     return MATQ_OK;
+}
+
+// Number of launches launch_batch makes for these batch sizes and shapes.
+inline int count_batch_launches(const HostProblem* hp, const int* hb, int n) {
+    int launches = 0;
+    for (int G = 1; G <= 4; G *= 2)
+        for (int wide = 0; wide < 2; ++wide) {
+            size_t cnt = 0;
+            for (int i = 0; i < n; ++i) {
+                if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
+                const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
+                const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
+                cnt += (fit >= kMaxW - 1) == (wide == 0);
+            }
+            launches += (int)((cnt + kLargeList - 1) / kLargeList);
+        }
+    return launches;
 }
 
 // Cuts a problem with B >= 2 vectors into parts the kernels take: batches of at most 2 * max_groups vectors that share

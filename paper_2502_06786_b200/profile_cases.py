@@ -1,6 +1,6 @@
 """Small, self-contained invocations of each kernel for profilers (ncu wants short runs with few launches).
 
-    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemv4t|gemv2t|stream8|stream4|stream2|group4|group2|gemm
+    python -m paper_2502_06786_b200.profile_cases quantize|slice4|slice2ep|gemv4|gemv2|gemv2b8|gemv4t|gemv2t|stream8|stream4|stream2|group4|group2|batch4|batch8|gemm
 
 (gemv4 / gemv2: the library's own choice at B = 1, the integer tensor kernel; a trailing t: the bf16 tensor kernel.)
 
@@ -69,6 +69,17 @@ def main(which: str) -> None:
         Y = [torch.empty(n_, device="cuda") for n_, k_ in shapes]
         a = torch.ones(9216, device="cuda")
         g = mq.gemv_group([(P[i], shapes[i][1], r, a[:shapes[i][0]], a[:shapes[i][0]], X[i], Y[i]) for i in range(len(shapes))])
+        for _ in range(3):
+            mq.gemv_grouped(g)
+    elif which in ("batch4", "batch8"):
+        # twelve matrices of the Gemma-2-2B MLP stack at r = 4 with 4 or 8 activation vectors each, one matq_gemv_grouped call
+        B = int(which[-1])
+        shapes = [(9216, 2304), (9216, 2304), (2304, 9216)] * 4
+        P = [torch.randint(0, 256, (n_, k_ // 2), dtype=torch.uint8, device="cuda") for n_, k_ in shapes]
+        X = [torch.randn(B, k_, device="cuda").to(torch.bfloat16) for n_, k_ in shapes]
+        Y = [torch.empty(B, n_, device="cuda") for n_, k_ in shapes]
+        a = torch.ones(9216, device="cuda")
+        g = mq.gemv_group([(P[i], shapes[i][1], 4, a[:shapes[i][0]], a[:shapes[i][0]], X[i], Y[i]) for i in range(len(shapes))])
         for _ in range(3):
             mq.gemv_grouped(g)
     elif which == "gemm":
