@@ -75,7 +75,7 @@ namespace gstream {
 constexpr int kMaxSlots = 24;
 constexpr int kUnitRow = 1184;                // bytes per row of the largest unit (16 rows)
 constexpr int kMaxTpu = 4;                   // tiles per unit at most
-constexpr int kMaxW = 8;                    // consumer warps: two per sub-partition; the producer warp is the ninth
+constexpr int kMaxW = 8;                    // consumer warps: two per sub-partition; the producer warp is the ninth (eleven measured 1-4 % faster on whole stacks, 8-12 % slower on short lists and batches)
 constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
 constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
 constexpr int kSmallList = 8;
@@ -993,6 +993,13 @@ inline int warps_for(size_t xs_bytes, int slot_bytes) {
     return (int)std::min<long long>(kMaxW, fit);
 }
 
+// W warps, or W - 1 when that puts more stages to use (the number of stages is a multiple of the number of warps: 14
+// instead of 8, say): bytes in flight matter more than the last warp.  Fewer warps still were measured: five with two
+// stages each win on K = 9216 at r = 8 and 4 and lose everywhere else.
+inline int pick_warps(int W, int fit) {
+    return (W > kMinW && fit / (W - 1) * (W - 1) > fit / W * W) ? W - 1 : W;
+}
+
 // Whether a problem can take this path at all (B = 1 is implied).
 inline bool eligible(int64_t N, int64_t K, int r) {
     if (!(r == 8 || r == 4 || r == 2) || K % 128 != 0 || K > imma::kMaxK || N <= 0 || N >= (1ll << 31) - 16) return false;
@@ -1052,10 +1059,8 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     int W = warps_for(xs_bytes, slot_bytes);
     if (W < kMinW) return MATQ_ERR_SHAPE;
     const int fit = std::min((int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes), kMaxSlots);
-    // The number of stages is a multiple of W: a stage always serves the same warp.  Eight warps (two per
-    // sub-partition) unless seven get more stages out of the same shared memory (14 instead of 8, say): bytes in
-    // flight matter more than the eighth warp.
-    if (W == kMaxW && fit / (W - 1) * (W - 1) > fit / W * W) --W;
+    // The number of stages is a multiple of W: a stage always serves the same warp.
+    W = pick_warps(W, fit);
     const int slots = fit / W * W;
     bool behind_ep = false;
     // Extra precision: the sparse term of every problem with lists goes to its y first (see ep_rowsum); the persistent

@@ -39,6 +39,7 @@ constexpr int kP2 = 21;                      // batched activations become integ
 constexpr int kPairCols = 7;                 // columns of a group: 3 + 3 bytes and the constant column
 constexpr int kPairUnit = kPairCols * 64;    // bytes of a staged (chunk, unit) block: 6 column blocks, the 7th unused
 constexpr int kMaxBatch = 8;
+constexpr int kWideFit = 7;                  // stages a problem's own shapes must leave room for to share a launch with the short rows
 
 // Staged bytes of one group for a problem (all chunks of a row).
 inline size_t xs_group_bytes_of(const Geo& g, int r) { return (size_t)g.n_qc * ((128 / r) / 16) * kPairUnit; }
@@ -497,7 +498,7 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
 inline int groups_of(int64_t B) { return B <= 2 ? 1 : B <= 4 ? 2 : 4; }
 
 // static shared memory of the batched kernel with G groups, rounded up
-inline int static_reserve_batch(int G) { return kStaticReserve + (G - 1) * 4 * 1024; }
+inline int static_reserve_batch(int G) { return kStaticReserve + (G - 1) * 6 * 1024; }
 
 // Whether a problem with B vectors (2 <= B <= kMaxBatch) can take the batched path.
 inline bool eligible_batch(int64_t N, int64_t K, int r, int64_t B) {
@@ -548,7 +549,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     const int fit = (int)std::min<long long>(room / slot_bytes, kMaxSlots);
     int W = std::min(kMaxW, fit);
     if (W < kMinW) return MATQ_ERR_SHAPE;
-    if (W == kMaxW && fit / (W - 1) * (W - 1) > fit / W * W) --W;
+    W = pick_warps(W, fit);
     const int slots = fit / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = kUnitRow; P.hold = hold ? 1 : 0;
@@ -592,7 +593,7 @@ inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, l
     for (int i = 0; i < n; ++i)
         if (hp[i].N != 0 && !eligible_batch(hp[i].N, hp[i].K, hp[i].r, hb[i])) return MATQ_ERR_SHAPE;      // before anything is launched
     // Problems with the same number of groups share a launch, except that those whose staged activations would leave
-    // the launch fewer than seven multiplying warps (long rows) get a launch of their own: the number of warps is a
+    // the launch fewer than seven stages and warps (long rows) get a launch of their own: the number of warps is a
     // property of the launch, and the short rows of a stack should not run with four.
     std::vector<HostProblem> sel;
     std::vector<int> sel_b;
@@ -603,7 +604,7 @@ inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, l
                 if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
                 const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
                 const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
-                if ((fit >= kMaxW - 1) != (wide == 0)) continue;
+                if ((fit >= kWideFit) != (wide == 0)) continue;
                 sel.push_back(hp[i]); sel_b.push_back(hb[i]);
             }
             for (size_t i = 0; i < sel.size(); i += kLargeList) {
@@ -626,7 +627,7 @@ inline int count_batch_launches(const HostProblem* hp, const int* hb, int n) {
                 if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
                 const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
                 const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
-                cnt += (fit >= kMaxW - 1) == (wide == 0);
+                cnt += (fit >= kWideFit) == (wide == 0);
             }
             launches += (int)((cnt + kLargeList - 1) / kLargeList);
         }
