@@ -315,6 +315,48 @@ __device__ __forceinline__ void multiply_unit(const unsigned char* wl_p, const u
 #undef MATQ_ITEM
 }
 
+// Two consecutive tiles of a unit at r = 2 in one pass: the B fragments of a chunk (four of the six 128-bit loads of an
+// r = 2 item) are loaded once and used for both tiles' weights.  Tile 0 accumulates in sets 0-3, tile 1 in sets 4-7; a
+// set is used again after eight MMAs.  `wl_p` / `wh_p` belong to tile 0, tile 1 lies `tile_bytes` further.
+__device__ __forceinline__ void multiply_two_tiles_r2(const unsigned char* wl_p, const unsigned char* wh_p, int tile_bytes, uint32_t x_sa, int xq_bytes,
+                                                      int col_lane, const uint4& cz, int n_chunks, int (&acc)[kSets][4]) {
+    uint4 xb[4];
+#pragma unroll
+    for (int m2 = 0; m2 < 4; ++m2) xb[m2] = cz;
+#pragma unroll 1
+    for (int c = 0; c < n_chunks; ++c) {
+        const uint4 wl0 = *reinterpret_cast<const uint4*>(wl_p + c * 64);
+        const uint4 wh0 = *reinterpret_cast<const uint4*>(wh_p + c * 64);
+        const uint4 wl1 = *reinterpret_cast<const uint4*>(wl_p + tile_bytes + c * 64);
+        const uint4 wh1 = *reinterpret_cast<const uint4*>(wh_p + tile_bytes + c * 64);
+#pragma unroll
+        for (int m2 = 0; m2 < 4; ++m2) lds128_if(xb[m2], x_sa + (uint32_t)(c * xq_bytes) + m2 * 256, col_lane);
+#pragma unroll
+        for (int m2 = 0; m2 < 4; ++m2) {
+#pragma unroll
+            for (int sub = 0; sub < 2; ++sub) {
+                const uint32_t b0 = sub ? xb[m2].z : xb[m2].x, b1 = sub ? xb[m2].w : xb[m2].y;
+#pragma unroll
+                for (int tile = 0; tile < 2; ++tile) {
+                    const uint4& wl = tile ? wl1 : wl0;
+                    const uint4& wh = tile ? wh1 : wh0;
+                    const uint32_t w_lo = m2 == 0 ? wl.x : m2 == 1 ? wl.y : m2 == 2 ? wl.z : wl.w;
+                    const uint32_t w_hi = m2 == 0 ? wh.x : m2 == 1 ? wh.y : m2 == 2 ? wh.z : wh.w;
+                    uint32_t a0, a1, a2, a3;
+                    if (sub == 0) {
+                        a0 = w_lo & 0x03030303u;  a2 = w_lo & 0x0f0f0f0fu;
+                        a1 = w_hi & 0x03030303u;  a3 = w_hi & 0x0f0f0f0fu;
+                    } else {
+                        a0 = w_lo & 0x3f3f3f3fu;  a2 = w_lo;
+                        a1 = w_hi & 0x3f3f3f3fu;  a3 = w_hi;
+                    }
+                    imma::mma_u8u8(acc[4 * tile + (2 * m2 + sub) % 4], a0, a1, a2, a3, b0, b1);
+                }
+            }
+        }
+    }
+}
+
 // Activation bytes of one problem in B-fragment order (all chunks of a row).  The byte layout is that of
 // gemv_imma.cuh; the values differ in one respect that saves a quarter (r = 2) or half (r = 4) of the mask
 // instructions of the multiply.  With V_i = round(x_i 2^(P - e - R i)) for the activation that meets field i of a
@@ -681,7 +723,9 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
     }
 }
 
-template <int NP>
+// PAIR2: the variant for lists whose problems are all at r = 2 (it processes two tiles of a unit per pass where it can;
+// the other lists keep the smaller kernel: the extra code costs them 1-2 %).
+template <int NP, bool PAIR2>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream(const __grid_constant__ Params<NP> P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -802,11 +846,24 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     multiply_item<2, 0>(wl_p + n_chunks * 64, wh_p + n_chunks * 64, x_sa + (uint32_t)(n_chunks * xq_bytes), col_lane, xt, acc);
                 }
             };
+            // r = 2, whole rows in a stage, no half-full chunk: two tiles of a unit per pass (see multiply_two_tiles_r2)
+            const bool pair_tiles = PAIR2 && R == 2 && G.contig && !half_tail;
+            auto multiply2 = [&](const unsigned char* tile_rows, int (&acc)[kSets][4]) {
+                const unsigned char* base = tile_rows + t * 16;
+                multiply_two_tiles_r2(base + (size_t)g * G.stride, base + (size_t)(g + 8) * G.stride, 16 * G.stride, x_sa0, xq_bytes, col_lane, cz, G.n_qc, acc);
+            };
             auto zero_acc = [&](int (&acc)[kSets][4]) {
 #pragma unroll
                 for (int c2 = 0; c2 < kSets; ++c2)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) acc[c2][i] = 0;
+            };
+            // after a pass over two tiles: tile 0's sets summed into acc[0], tile 1's into acc[4]
+            auto fold_two = [&](int (&acc)[kSets][4]) {
+#pragma unroll
+                for (int c2 = 1; c2 < 4; ++c2)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { acc[0][i] += acc[c2][i]; acc[4][i] += acc[4 + c2][i]; }
             };
             auto fold = [&](int (&acc)[kSets][4]) {
 #pragma unroll
@@ -923,14 +980,18 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 const unsigned char* rows = ring + (size_t)slot * P.slot_bytes;
                 const bool tile_done = !pl.split && pn == G.n_panels - 1;
                 for (int k = 0; k < n_tiles; ++k) {
+                    const bool two = pair_tiles && k + 1 < n_tiles;       // this tile and the next in one pass
                     if (k > 0) zero_acc(acc);
-                    if (landed) multiply(rows + (size_t)k * 16 * G.stride, pn, acc);
-                    if (k == n_tiles - 1) {                               // the last read of the stage is done
+                    if (landed) {
+                        if (two) multiply2(rows + (size_t)k * 16 * G.stride, acc);
+                        else multiply(rows + (size_t)k * 16 * G.stride, pn, acc);
+                    }
+                    if (k + (two ? 1 : 0) == n_tiles - 1) {               // the last read of the stage is done
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&s_empty[slot]));
                     }
                     if (tile_done) {
-                        fold(acc);
+                        if (two) fold_two(acc); else fold(acc);
                         if (ep && !epv_ok) {                                  // not loaded a round ahead: wait for the sums, load them now
                             await_ep();
 #pragma unroll
@@ -941,6 +1002,11 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                         finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
                                     k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3],
                                     k == 0 ? epv[0] : k == 1 ? epv[1] : k == 2 ? epv[2] : epv[3], lane, !*abort_flag);
+                        if (two) {
+                            ++k;
+                            finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[4][0], acc[4][1], acc[4][2], acc[4][3],
+                                        k == 1 ? sc[1] : sc[3], k == 1 ? epv[1] : epv[3], lane, !*abort_flag);
+                        }
                     }
                 }
                 if (n_tiles == 0) {
@@ -1022,7 +1088,7 @@ inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, co
 
 template <int NP>
 inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
-    static std::atomic<unsigned long long> smem_ok{0};
+    static std::atomic<unsigned long long> smem_ok{0}, smem_ok2{0};
     Params<NP> P;
     long long items = 0, tiles = 0;
     for (int i = 0; i < n; ++i) {
@@ -1099,8 +1165,10 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     }
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
-    auto kern = gemv_stream<NP>;
-    if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
+    bool all_r2 = true;
+    for (int i = 0; i < m; ++i) all_r2 = all_r2 && P.p[i].r == 2;
+    auto kern = all_r2 ? gemv_stream<NP, true> : gemv_stream<NP, false>;
+    if (!opt_in_max_smem(kern, all_r2 ? smem_ok2 : smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)((W + 1) * 32));
