@@ -297,6 +297,14 @@ class DeviceStack:
                 mq.slice_pack(self.q[i], 2, extra_precision=True, packed=self.p2[i], ovf_row_ptr=self.rp[i],
                               ovf_col=self.col[i], ovf_capacity=self.cap[i], ovf_count=self.cnt[i], dev_status=self.status)
 
+        def sp42():
+            for i in range(n):
+                mq.slice_pack_nested(self.q[i], extra_precision=True, packed4=self.p4[i], packed2=self.p2[i], ovf_row_ptr=self.rp[i],
+                                     ovf_col=self.col[i], ovf_capacity=self.cap[i], ovf_count=self.cnt[i], dev_status=self.status)
+        self.slice_alone = {"slice_pack_r4_alone": (sp4, n, sum(bytes_slice_pack(N, K, 4) for (_, _, _, N, K) in S)),
+                            "slice_pack_r2_ep_alone": (sp2, 2 * n, sum(bytes_slice_pack(N, K, 2, z) for (_, _, _, N, K), z in
+                                                                       zip(S, getattr(self, "nnz", [0] * n))))}
+
         def gemv_b8(nm, r):
             """B = 8 over the whole stack in one matq_gemv_grouped call."""
             g = self.problems(nm, r, False, list(range(n)), batch=True)
@@ -311,8 +319,9 @@ class DeviceStack:
         gep, lep = self.gemv_b1("g2ep", 2, True, n)
         return [
             ("quantize", quant, n, sum(bytes_quantize(N, K) for (_, _, _, N, K) in S)),
-            ("slice_pack_r4", sp4, n, sum(bytes_slice_pack(N, K, 4) for (_, _, _, N, K) in S)),
-            ("slice_pack_r2_ep", sp2, 2 * n, sum(bytes_slice_pack(N, K, 2, z) for (_, _, _, N, K), z in zip(S, nnz))),
+            # the int4 and the int2 plane (+ lists) from one read of the codes: the codes count once
+            ("slice_pack_r4_r2_ep", sp42, 2 * n, sum(bytes_slice_pack(N, K, 4) + bytes_slice_pack(N, K, 2, z) - N * K
+                                                     for (_, _, _, N, K), z in zip(S, nnz))),
             # the decode stages come last, the B = 1 ones after the B = 8 ones: a stage that directly follows slice_pack
             # also pays the write-back of the planes that stage left dirty in the L2, which no decode loop ever sees
             ("gemv_r4_b8", *gemv_b8("g4b8", 4), sum(bytes_gemv(N, K, 4, 8) for (_, _, _, N, K) in S)),
@@ -448,6 +457,9 @@ def run_cuda(args, rank, world, local_rank):
             ms = time_graph(torch, capture(torch, fn))
             stages[f"{key}_{label}"] = dict(gemv_entry(ms, nbytes, peaks, launches), in_step=False)
             gemv_frac[f"cfg2_{key[5:]}_{label}"] = stages[f"{key}_{label}"]["frac_hbm"]
+    for key, (fn, launches, nbytes) in st.slice_alone.items():          # the two planes by separate calls, for comparison
+        ms = time_graph(torch, capture(torch, fn))
+        stages[key] = dict(gemv_entry(ms, nbytes, peaks, launches), in_step=False)
     for nm, r, key in (("g4b8", 4, "gemv_r4_b8"), ("g2b8", 2, "gemv_r2_b8")):
         gemv_frac[f"cfg2_{key[5:]}_whole_stack_call"] = stages[key]["frac_hbm"]
         fn, launches = st.gemv_b8_per_matrix(nm, r)
@@ -500,7 +512,7 @@ def run_cuda(args, rank, world, local_rank):
             "data": "synthetic",
             "config": {"workload": f"configs[1] Gemma-2-2B-shaped MLP decode stack, {args.layers} layers x (gate,up 9216x2304; down 2304x9216), "
                                    "bf16 N(0,0.02) weights, x bf16 N(0,1)",
-                       "step": "quantize -> slice_pack r=4 -> slice_pack r=2 + extra-precision lists -> gemv r=4, r=2 at B=8 -> gemv r=4, r=2, r=2 E.P. at B=1 "
+                       "step": "quantize -> slice_pack r=4 and r=2 + extra-precision lists in one pass (matq_slice_pack_nested) -> gemv r=4, r=2 at B=8 -> gemv r=4, r=2, r=2 E.P. at B=1 "
                                "(all decode stages: matq_gemv_grouped, whole stack per call)"
                                "; dense multi-precision forward measured separately (gemm_multi_cfg4)",
                        "value_definition": "decode GEMV at B = 1: algorithmic HBM bytes of the gemv_r4_b1 and gemv_r2_b1 stages / their device time "

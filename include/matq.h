@@ -160,6 +160,20 @@ int matq_slice_pack(const uint8_t *q, int64_t N, int64_t K, int c, int r, int ex
                     int32_t *dev_status, void *stream);
 
 /*
+ * (2b) The int4 and the int2 plane of a nested model from ONE read of its int8 codes (Section 3.2: every nested
+ *      precision is a slice of the same c-bit code): exactly matq_slice_pack(r = 4) into packed4 (Eq. 6) and
+ *      matq_slice_pack(r = 2, extra_precision) into packed2 with its overflow lists (Eq. 6, or Eq. 8's base plane and
+ *      lists), bit for bit, at 1.75 instead of 2.75 bytes of HBM traffic per weight.  One kernel when K % 16 == 0,
+ *      K <= 16384, N * K < 2^31, the buffers are 16-byte aligned and extra_precision is set; two calls otherwise.
+ *   packed4   out  uint8 [N, K / 2]        packed2   out  uint8 [N, K / 4]       (K % 4 == 0)
+ *   the overflow arguments, dev_status and the error behaviour are those of matq_slice_pack for r = 2.
+ */
+int matq_slice_pack_nested(const uint8_t *q, int64_t N, int64_t K, int c, uint8_t *packed4, uint8_t *packed2,
+                           int extra_precision,
+                           int32_t *ovf_row_ptr, uint16_t *ovf_col, int64_t ovf_capacity, int64_t *ovf_count,
+                           int32_t *dev_status, void *stream);
+
+/*
  * (3) Decode-time weight-only quantised linear layer on a packed r-bit plane:
  *       y[b,n] = sum_k x[b,k] * alpha_n * (S[n,k] - z_n),   S = k << (c - r)
  *     (dequantisation alpha * (S - z) with the same alpha, z at every r, since

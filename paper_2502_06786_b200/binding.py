@@ -24,7 +24,7 @@ GEMV_TEST_STALL = 0x8000
 TEACHER_AND_TARGET = 256    # matq_gemm_multi_loss: teacher[i] = TEACHER_AND_TARGET + j
 
 EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_quantize", "matq_quantize_clip",
-           "matq_slice_pack", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped", "matq_gemv_grouped_launches",
+           "matq_slice_pack", "matq_slice_pack_nested", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped", "matq_gemv_grouped_launches",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
            "matq_gemm_multi_loss_workspace_bytes", "matq_gemm_multi_loss",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
@@ -61,6 +61,8 @@ def _load():
     lib.matq_quantize_clip.argtypes = [vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.matq_slice_pack.restype = i32
     lib.matq_slice_pack.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.matq_slice_pack_nested.restype = i32
+    lib.matq_slice_pack_nested.argtypes = [vp, i64, i64, i32, vp, vp, i32, vp, vp, i64, vp, vp, vp]
     lib.matq_gemv_workspace_bytes.restype = sz
     lib.matq_gemv_workspace_bytes.argtypes = [i64, i64, i32, i32]
     lib.matq_gemv.restype = i32
@@ -192,6 +194,34 @@ def slice_pack(q, r, extra_precision=False, packed=None, sliced_unpacked=None, o
     _check(st, "matq_slice_pack", raise_on_error)
     return dict(status=st, packed=packed, sliced=sliced_unpacked, ovf_row_ptr=ovf_row_ptr, ovf_col=ovf_col,
                 ovf_count=ovf_count)
+
+
+def slice_pack_nested(q, extra_precision=True, packed4=None, packed2=None, ovf_row_ptr=None, ovf_col=None, ovf_capacity=None,
+                      ovf_count=None, dev_status=None, c=8, raise_on_error=True):
+    """matq_slice_pack_nested.  Returns dict(status, packed4, packed2, ovf_row_ptr, ovf_col, ovf_count)."""
+    _dev(q, torch.uint8, "q", 2)
+    if not q.is_contiguous():
+        raise ValueError("q must be contiguous")
+    N, K = q.shape
+    dev = q.device
+    if packed4 is None:
+        packed4 = torch.empty((N, K // 2), dtype=torch.uint8, device=dev)
+    if packed2 is None:
+        packed2 = torch.empty((N, K // 4), dtype=torch.uint8, device=dev)
+    if extra_precision:
+        if ovf_row_ptr is None:
+            ovf_row_ptr = torch.empty(N + 1, dtype=torch.int32, device=dev)
+        if ovf_capacity is None:
+            ovf_capacity = ovf_col.numel() if ovf_col is not None else N * K
+        if ovf_col is None:
+            ovf_col = torch.empty(max(ovf_capacity, 1), dtype=torch.uint16, device=dev)
+        if ovf_count is None:
+            ovf_count = torch.zeros(1, dtype=torch.int64, device=dev)
+    st = _lib.matq_slice_pack_nested(_ptr(q), N, K, c, _ptr(packed4), _ptr(packed2), int(bool(extra_precision)),
+                                     _ptr(ovf_row_ptr), _ptr(ovf_col), int(ovf_capacity or 0), _ptr(ovf_count),
+                                     _ptr(dev_status), _stream())
+    _check(st, "matq_slice_pack_nested", raise_on_error)
+    return dict(status=st, packed4=packed4, packed2=packed2, ovf_row_ptr=ovf_row_ptr, ovf_col=ovf_col, ovf_count=ovf_count)
 
 
 def gemv_workspace_bytes(N, K, r, B) -> int:

@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(256) ep_init_flags(uint32_t* __restrict__ row_
 template <int PACK_R>
 __global__ void __launch_bounds__(1024)
 slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, int rows_per_warp,
-              uint8_t* __restrict__ packed, uint8_t* __restrict__ sliced, uint32_t* __restrict__ row_ptr,
+              uint8_t* __restrict__ packed, uint8_t* __restrict__ packed4, uint8_t* __restrict__ sliced, uint32_t* __restrict__ row_ptr,
               uint16_t* __restrict__ ovf_col, int64_t capacity, int64_t* __restrict__ total_out, int32_t* dev_status) {
     extern __shared__ __align__(16) uint8_t ep_smem[];
     __shared__ uint32_t base_s, total_s;
@@ -357,6 +357,11 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
                             slice_pack4_r2(v[u].x, b0, m0); slice_pack4_r2(v[u].y, b1, m1);
                             slice_pack4_r2(v[u].z, b2, m2); slice_pack4_r2(v[u].w, b3, m3);
                             reinterpret_cast<uint32_t*>(packed)[c_row + c] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+                            if (packed4) {                      // the int4 plane of the same codes from the same read (Eq. 6)
+                                const uint32_t k0 = slice4(v[u].x, 4).k, k1 = slice4(v[u].y, 4).k, k2 = slice4(v[u].z, 4).k, k3 = slice4(v[u].w, 4).k;
+                                reinterpret_cast<uint2*>(packed4)[c_row + c] =
+                                    make_uint2(pack4<4>(k0) | (pack4<4>(k1) << 16), pack4<4>(k2) | (pack4<4>(k3) << 16));
+                            }
                             const uint32_t m = m0 | (m1 << 4) | (m2 << 8) | (m3 << 12);
                             mrow[c] = (uint16_t)m;
                             cnt += __popc(m);
@@ -508,7 +513,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
 // Returns MATQ_ERR_SHAPE when no tile fits the shared-memory budget (the caller then uses the three-kernel chain).
 template <int PACK_R>
 int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, uint8_t* sliced, int32_t* row_ptr,
-              uint16_t* ovf_col, int64_t capacity, int64_t* total, int32_t* dev_status, cudaStream_t s) {
+              uint16_t* ovf_col, int64_t capacity, int64_t* total, int32_t* dev_status, cudaStream_t s, uint8_t* packed4 = nullptr) {
     const int sms = sm_count();
     const size_t row_smem = sizeof(int) + (size_t)(K / 16) * sizeof(uint16_t);
     int nwarps = 32, rpw = 1;
@@ -547,7 +552,7 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     cfg.numAttrs = 1;
     const int K32 = (int)K;
     uint32_t* flags = reinterpret_cast<uint32_t*>(row_ptr);
-    if (cudaLaunchKernelEx(&cfg, slice_pack_ep<PACK_R>, q, N, K32, r, rpw, packed, sliced, flags, ovf_col, capacity, total,
+    if (cudaLaunchKernelEx(&cfg, slice_pack_ep<PACK_R>, q, N, K32, r, rpw, packed, packed4, sliced, flags, ovf_col, capacity, total,
                            dev_status) != cudaSuccess) {
         cudaGetLastError();
         return MATQ_ERR_CUDA;
@@ -634,4 +639,25 @@ extern "C" int matq_slice_pack(const uint8_t* q, int64_t N, int64_t K, int c, in
         else ovf_fill<<<(unsigned)blocks, kSliceThreads, 0, s>>>(q, N, K, r, ovf_row_ptr, ovf_count, ovf_capacity, ovf_col);
     }
     return launch_status();
+}
+
+extern "C" int matq_slice_pack_nested(const uint8_t* q, int64_t N, int64_t K, int c, uint8_t* packed4, uint8_t* packed2, int extra_precision,
+                                      int32_t* ovf_row_ptr, uint16_t* ovf_col, int64_t ovf_capacity, int64_t* ovf_count,
+                                      int32_t* dev_status, void* stream) {
+    using namespace matq;
+    if (N < 0 || K <= 0 || (!q && N > 0) || !packed4 || !packed2) return MATQ_ERR_INVALID_ARG;
+    if (c != kCodeBits) return MATQ_ERR_UNSUPPORTED;
+    if (K % 4 != 0) return MATQ_ERR_SHAPE;
+    if (extra_precision && (!ovf_row_ptr || !ovf_col || !ovf_count || ovf_capacity < 0)) return MATQ_ERR_INVALID_ARG;
+    if (extra_precision && K > 65536) return MATQ_ERR_SHAPE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // one pass over the codes when the one-pass extra-precision kernel takes the shape; two calls otherwise
+    const bool vec = (K % 16 == 0) && aligned16(q) && aligned16(packed4) && aligned16(packed2);
+    if (extra_precision && N > 0 && vec && K <= 16384 && N * K < (int64_t(1) << 31)) {
+        const int st = launch_ep<2>(q, N, K, 2, packed2, nullptr, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, s, packed4);
+        if (st != MATQ_ERR_SHAPE) return st;
+    }
+    const int st = matq_slice_pack(q, N, K, c, 4, 0, packed4, nullptr, nullptr, nullptr, 0, nullptr, dev_status, stream);
+    if (st != MATQ_OK) return st;
+    return matq_slice_pack(q, N, K, c, 2, extra_precision, packed2, nullptr, ovf_row_ptr, ovf_col, ovf_capacity, ovf_count, dev_status, stream);
 }

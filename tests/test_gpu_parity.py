@@ -208,6 +208,39 @@ def test_extra_precision_lists_bit_exact(r, N, K, p):
     assert torch.equal(std["packed"], out["packed"])
 
 
+@pytest.mark.parametrize("ep", [True, False])
+@pytest.mark.parametrize("N,K,p", [(64, 2304, 0.05), (1500, 512, 0.125), (9, 1000, 0.3), (40, 4096, 0.0), (33, 16384, 0.05),
+                                   (12, 32768, 0.02), (10, 16, 0.3), (9216, 2304, 0.005), (4099, 256, 0.1), (7, 20, 0.2)])
+def test_slice_pack_nested_bit_exact(N, K, p, ep):
+    # the int4 and the int2 plane (+ Eq. 8 lists) from one read of the codes: the bits of the two single calls and of
+    # the oracle; shapes the one-pass kernel takes, and shapes that fall back to two calls (K % 16 != 0, K > 16384)
+    q = synth.skewed_codes((N, K), p, 224, 900 + N) if p > 0 else synth.uniform_codes((N, K), 1) // 2
+    if N > 8:
+        q[3, :] = 255
+        q[5, :] = 0
+    status = status_word()
+    out = mq.slice_pack_nested(dev(q), extra_precision=ep, dev_status=status)
+    want4 = ref.slice_pack(q, 4)
+    want2 = ref.slice_pack(q, 2, extra_precision=ep)
+    assert np.array_equal(host(out["packed4"]), want4["packed"])
+    assert np.array_equal(host(out["packed2"]), want2["packed"])
+    if ep:
+        cnt = int(host(out["ovf_count"])[0])
+        assert cnt == want2["ovf_count"]
+        assert np.array_equal(host(out["ovf_row_ptr"]), want2["ovf_row_ptr"])
+        assert np.array_equal(host(out["ovf_col"])[:cnt], want2["ovf_col"])
+    assert int(host(status)[0]) == mq.OK
+
+
+def test_slice_pack_nested_argument_errors():
+    q = dev(synth.uniform_codes((8, 64), 3))
+    p4 = torch.empty((8, 32), dtype=torch.uint8, device="cuda")
+    st = mq._lib.matq_slice_pack_nested(q.data_ptr(), 8, 64, 8, p4.data_ptr(), None, 0, None, None, 0, None, None, None)
+    assert st == mq.ERR_INVALID_ARG
+    out = mq.slice_pack_nested(dev(synth.uniform_codes((8, 6), 3)), raise_on_error=False)
+    assert out["status"] == mq.ERR_SHAPE
+
+
 def test_extra_precision_capacity_error_is_a_status():
     q = synth.skewed_codes((32, 512), 0.2, 224, 77)
     want = ref.slice_pack(q, 2, extra_precision=True)
