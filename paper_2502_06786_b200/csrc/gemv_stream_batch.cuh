@@ -19,7 +19,7 @@
 // again after eight MMAs, as in the single-vector kernel.
 //
 // Staging.  The activations of the current problem are kept in shared memory as byte units in B-fragment order, one
-// region per group: per (chunk, 16-weight unit) seven column blocks of 64 bytes (bytes 0-2 of the first vector, 0-2 of
+// region per group: per (chunk, 16-weight unit) six column blocks of 64 bytes (bytes 0-2 of the first vector, 0-2 of
 // the second; the constant column is held in registers by the lanes of column 6).  A CTA converts only the problems
 // its share of the list touches (one or two when a call covers a whole decoder stack), which is what makes batches
 // affordable here: a kernel per matrix has every CTA convert all B vectors for every matrix.
@@ -37,7 +37,7 @@ namespace gstream {
 
 constexpr int kP2 = 21;                      // batched activations become integers below 2^(kP2 + 1)
 constexpr int kPairCols = 7;                 // columns of a group: 3 + 3 bytes and the constant column
-constexpr int kPairUnit = kPairCols * 64;    // bytes of a staged (chunk, unit) block: 6 column blocks, the 7th unused
+constexpr int kPairUnit = (kPairCols - 1) * 64;   // bytes of a staged (chunk, unit) block: the six byte columns (the constant column lives in registers)
 constexpr int kMaxBatch = 8;
 constexpr int kWideFit = 7;                  // stages a problem's own shapes must leave room for to share a launch with the short rows
 
