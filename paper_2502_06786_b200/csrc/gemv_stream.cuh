@@ -75,7 +75,10 @@ namespace gstream {
 constexpr int kMaxSlots = 24;
 constexpr int kUnitRow = 1184;                // bytes per row of the largest unit (16 rows)
 constexpr int kMaxTpu = 4;                   // tiles per unit at most
-constexpr int kMaxW = 8;                    // consumer warps: two per sub-partition; the producer warp is the ninth (eleven measured 1-4 % faster on whole stacks, 8-12 % slower on short lists and batches)
+constexpr int kMaxW = 11;                   // consumer warps at most (with the producer: 12 warps, 168 registers a thread)
+constexpr int kFewW = 8;                    // ... on lists with little work per CTA and for batches: two per sub-partition
+constexpr int kManyItems = 1000;            // items per CTA from which a list gets kMaxW warps: eleven warps measured 1-4 %
+                                            // faster on whole decoder stacks and 8-12 % slower on a layer's three matrices
 constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
 constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
 constexpr int kSmallList = 8;
@@ -1122,7 +1125,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         ++m;
     }
     for (int i = m; i < NP; ++i) P.p[i] = Problem{};
-    int W = warps_for(xs_bytes, slot_bytes);
+    int W = std::min(warps_for(xs_bytes, slot_bytes), items / grid >= kManyItems ? kMaxW : kFewW);
     if (W < kMinW) return MATQ_ERR_SHAPE;
     const int fit = std::min((int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes), kMaxSlots);
     // The number of stages is a multiple of W: a stage always serves the same warp.

@@ -547,7 +547,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     xs_bytes = (xs_bytes + 127) / 128 * 128;
     const long long room = (long long)kSmemLimit - static_reserve_batch(G) - (long long)xs_bytes;
     const int fit = (int)std::min<long long>(room / slot_bytes, kMaxSlots);
-    int W = std::min(kMaxW, fit);
+    int W = std::min(kFewW, fit);
     if (W < kMinW) return MATQ_ERR_SHAPE;
     W = pick_warps(W, fit);
     const int slots = fit / W * W;
