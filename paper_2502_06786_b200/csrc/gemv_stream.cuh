@@ -576,7 +576,16 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
     if (P.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;");
     const long long lo = P.rows * blockIdx.x / gridDim.x, hi = P.rows * (blockIdx.x + 1) / gridDim.x;
-    for (int p = 0; p < P.n; ++p) {
+    int p_first = 0;
+    {
+        int a = 0, b = P.n - 1;                                           // last problem that starts at or before lo
+        while (a < b) {
+            const int m = (a + b + 1) >> 1;
+            if (P.p[m].row0 <= lo) a = m; else b = m - 1;
+        }
+        p_first = a;
+    }
+    for (int p = p_first; p < P.n && P.p[p].row0 < hi; ++p) {           // only the problems this CTA's rows belong to
         const EpProblem& pr = P.p[p];
         const long long a = lo > pr.row0 ? lo - pr.row0 : 0;
         const long long b = hi - pr.row0 < pr.N ? hi - pr.row0 : pr.N;
@@ -585,13 +594,26 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
         if (tid == 0) s_nlong = 0;
         for (int i = tid; i < (pr.K >> 3); i += kEpThreads) reinterpret_cast<uint4*>(xs)[i] = ld_x4(pr.x + 8 * i);
         __syncthreads();
-        // two rows per group and pass: their dependent loads (row_ptr, then columns, then the gathers) overlap.
-        // A row lists at most K columns: row_ptr values that say otherwise are cut short, so that every loop ends.
-        for (long long row = a + grp; row < b; row += 2 * (kEpThreads / 8)) {
+        // Two rows per group and pass.  What a pass costs is dependent round trips to the L2 / HBM, so they are kept to
+        // one: the list bounds of the NEXT pass are requested before this pass's columns, and the first four columns of
+        // each lane (32 entries of a row; most rows have fewer) are requested together for both rows, predicated, before
+        // any is used.  A row lists at most K columns: row_ptr values that say otherwise are cut short, so that every
+        // loop ends.
+        auto bounds = [&](long long r, bool on, int& lo_e, int& hi_e) {
+            lo_e = on ? max(pr.row_ptr[r], 0) : 0;
+            hi_e = on ? min(pr.row_ptr[r + 1], lo_e + pr.K) : 0;
+        };
+        auto xat = [&](int c) { return c < 0 ? 0.f : __bfloat162float(xs[c < pr.K ? c : c % pr.K]); };
+        constexpr int kStride = 2 * (kEpThreads / 8);
+        int e0, e1, f0, f1;
+        bounds(a + grp, a + grp < b, e0, e1);
+        bounds(a + grp + kEpThreads / 8, a + grp + kEpThreads / 8 < b, f0, f1);
+        for (long long row = a + grp; row < b; row += kStride) {
             const long long row2 = row + kEpThreads / 8;
             const bool two = row2 < b;
-            const int e0 = max(pr.row_ptr[row], 0), e1 = min(pr.row_ptr[row + 1], e0 + pr.K);
-            const int f0 = two ? max(pr.row_ptr[row2], 0) : 0, f1 = two ? min(pr.row_ptr[row2 + 1], f0 + pr.K) : 0;
+            int ne0, ne1, nf0, nf1;                                        // the next pass's lists
+            bounds(row + kStride, row + kStride < b, ne0, ne1);
+            bounds(row2 + kStride, row2 + kStride < b, nf0, nf1);
             const bool long_a = e1 - e0 > kEpLongList, long_b = f1 - f0 > kEpLongList;
             bool defer_a = false, defer_b = false;
             if (long_a || long_b) {                                       // remembered for the CTA-wide pass below
@@ -607,8 +629,17 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
                 defer_a = long_a && slot_a < kEpMaxLong;
                 defer_b = long_b && slot_b < kEpMaxLong;
             }
-            float sa = defer_a ? 0.f : ep_partial(pr.col, xs, pr.K, e0, e1, sub, 8);
-            float sb = (!two || defer_b) ? 0.f : ep_partial(pr.col, xs, pr.K, f0, f1, sub, 8);
+            const int ea = defer_a ? e0 : e1, eb = (!two || defer_b) ? f0 : f1;   // an empty range for rows not summed here
+            int ca[4], cb[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                ca[j] = e0 + sub + 8 * j < ea ? (int)pr.col[e0 + sub + 8 * j] : -1;
+                cb[j] = f0 + sub + 8 * j < eb ? (int)pr.col[f0 + sub + 8 * j] : -1;
+            }
+            float sa = (xat(ca[0]) + xat(ca[1])) + (xat(ca[2]) + xat(ca[3]));
+            float sb = (xat(cb[0]) + xat(cb[1])) + (xat(cb[2]) + xat(cb[3]));
+            if (ea - e0 > 32) sa += ep_partial(pr.col, xs, pr.K, e0 + 32, ea, sub, 8);
+            if (eb - f0 > 32) sb += ep_partial(pr.col, xs, pr.K, f0 + 32, eb, sub, 8);
             sa += __shfl_xor_sync(gmask, sa, 4);  sb += __shfl_xor_sync(gmask, sb, 4);   // the eight lanes of this group only: the
             sa += __shfl_xor_sync(gmask, sa, 2);  sb += __shfl_xor_sync(gmask, sb, 2);   // other groups of the warp may already have
             sa += __shfl_xor_sync(gmask, sa, 1);  sb += __shfl_xor_sync(gmask, sb, 1);   // left the loop
@@ -616,6 +647,7 @@ ep_rowsum(const __grid_constant__ EpParams<NP> P) {
                 if (!defer_a) pr.y[row] = sa;
                 if (two && !defer_b) pr.y[row2] = sb;
             }
+            e0 = ne0; e1 = ne1; f0 = nf0; f1 = nf1;
         }
         __syncthreads();
         // long lists (a row whose codes all sit in the extra bucket lists K columns): all threads on one row at a time
@@ -1152,7 +1184,9 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
             auto ek = ep_rowsum<NP>;
             if (!opt_in_max_smem(ek, ep_smem_ok)) return MATQ_ERR_CUDA;
             cudaLaunchConfig_t ec = {};
-            ec.gridDim = dim3((unsigned)std::max<long long>(1, std::min<long long>(4ll * sms, (rows + 63) / 64)));
+            int per_sm = 0;                                  // one wave: as many CTAs as are resident together
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ek, kEpThreads, (size_t)2 * k_max) != cudaSuccess || per_sm < 1) per_sm = 1;
+            ec.gridDim = dim3((unsigned)std::max<long long>(1, std::min<long long>((long long)per_sm * sms, (rows + 63) / 64)));
             ec.blockDim = dim3(kEpThreads);
             ec.dynamicSmemBytes = (size_t)2 * k_max;
             ec.stream = s;
