@@ -99,14 +99,14 @@ struct Problem {
     int N, K;
     int r;
     int B;                    // activation vectors (1 in gemv_stream; 2 .. 8 in gemv_stream_batch)
-    long long item0;          // (tile x chunk) items of the problems before this one
+    long long item0;          // cost (tile_cost units) of the problems before this one
 };
 
 template <int NP>
 struct Params {
     CUtensorMap tm[NP];       // over each plane as [N][row_bytes / 8] 64-bit words, box 16 x panel (only read for long rows)
     Problem p[NP];
-    long long items;          // total items
+    long long items;          // total cost of the list (tile_cost units: sixteenths of an item)
     long long wait_cycles;    // limit of a wait, in SM clock cycles
     int32_t* dev_status;
     int n;                    // problems
@@ -152,6 +152,12 @@ __host__ __device__ inline Geo geometry(int N, int K, int r, int unit_row) {
     g.stride = g.panel_qc * 64;
     return g;
 }
+
+// What a tile of a problem counts for when the list is divided among the CTAs, in sixteenths of a (tile x chunk) item:
+// the list is cut into shares of equal COST, not of equal bytes.  Rows of four or more K panels cost the multiplying
+// warps an eighth more per byte at r = 4 and r = 2 (measured: 9216-wide rows run at 0.78 / 0.56 of the HBM rate where
+// 2304-wide rows run at 0.89 / 0.64); at r = 8 every shape is bound by HBM and a byte is a byte.
+__host__ __device__ inline int tile_cost(const Geo& g, int r) { return g.n_qc * ((g.n_panels >= 4 && r != 8) ? 18 : 16); }
 
 // How a CTA's share of a problem (T tiles, i.e. ceil(T / tpu) groups of tiles) is laid out as a sequence of units.
 // Unit s goes to warp s mod W; the sequence is padded with empty units to a multiple of W.
@@ -230,8 +236,9 @@ __device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, 
         const long long i0 = P.p[p].item0;
         if (i0 >= hi) return false;
         const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r, P.unit_row);
-        const long long a = lo > i0 ? (lo - i0 + g.n_qc - 1) / g.n_qc : 0;
-        const long long b = (hi - i0 + g.n_qc - 1) / g.n_qc;
+        const int tc = tile_cost(g, P.p[p].r);
+        const long long a = lo > i0 ? (lo - i0 + tc - 1) / tc : 0;
+        const long long b = (hi - i0 + tc - 1) / tc;
         ++p;
         t_lo = (int)(a < g.tiles ? a : g.tiles);
         t_hi = (int)(b < g.tiles ? b : g.tiles);
@@ -1130,7 +1137,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         if (hp[i].N == 0) continue;
         if (!eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;
         const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-        items += (long long)g.tiles * g.n_qc;
+        items += (long long)g.tiles * tile_cost(g, hp[i].r);
         tiles += g.tiles;
     }
     if (tiles == 0) return MATQ_OK;
@@ -1151,13 +1158,13 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         q.item0 = item0;
         const Geo g = geometry(q.N, q.K, q.r, unit_row);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
-        item0 += (long long)g.tiles * g.n_qc;
+        item0 += (long long)g.tiles * tile_cost(g, q.r);
         xs_bytes = std::max(xs_bytes, xs_bytes_of(g, q.r));
         slot_bytes = std::max(slot_bytes, slot_bytes_of(g));
         ++m;
     }
     for (int i = m; i < NP; ++i) P.p[i] = Problem{};
-    int W = std::min(warps_for(xs_bytes, slot_bytes), items / grid >= kManyItems ? kMaxW : kFewW);
+    int W = std::min(warps_for(xs_bytes, slot_bytes), items / grid >= 16ll * kManyItems ? kMaxW : kFewW);
     if (W < kMinW) return MATQ_ERR_SHAPE;
     const int fit = std::min((int)((kSmemLimit - kStaticReserve - xs_bytes) / slot_bytes), kMaxSlots);
     // The number of stages is a multiple of W: a stage always serves the same warp.

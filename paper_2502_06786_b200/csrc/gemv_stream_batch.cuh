@@ -519,7 +519,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     for (int i = 0; i < n; ++i) {
         if (hp[i].N == 0) continue;
         const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-        items += (long long)g.tiles * g.n_qc;
+        items += (long long)g.tiles * tile_cost(g, hp[i].r);
         tiles += g.tiles;
     }
     if (tiles == 0) return MATQ_OK;
@@ -538,7 +538,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
         q.item0 = item0;
         const Geo g = geometry(q.N, q.K, q.r, kUnitRow);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
-        item0 += (long long)g.tiles * g.n_qc;
+        item0 += (long long)g.tiles * tile_cost(g, q.r);
         xs_bytes = std::max(xs_bytes, (size_t)G * xs_group_bytes_of(g, q.r));
         slot_bytes = std::max(slot_bytes, slot_bytes_of(g));
         ++m;
