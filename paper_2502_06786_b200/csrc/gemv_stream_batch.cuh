@@ -232,7 +232,8 @@ __device__ __forceinline__ void multiply_unit_pair(const unsigned char* wl_p, co
     constexpr int kM2 = (128 / R) / 16;
     constexpr int kFrag = 2 * kM2;                                   // fragments of an item
     constexpr int kS = kSets / G;
-    constexpr int kU = kS > kFrag ? kS / kFrag : 1;                  // items per round: a round uses every set of a group
+    constexpr int kU = kS > kFrag ? kS / kFrag : (R == 8 ? 2 : 1);   // items per round: a round uses every set of a group; at r = 8 at least
+                                                                     // two, so that the loads of the second item are in flight during the first's MMAs
 #define MATQ_PITEM(I) multiply_item_pair<R, G, ((I) * kFrag) % kS>(wl_p + (c + (I)) * 64, wh_p + (c + (I)) * 64, x_sa + (uint32_t)((c + (I)) * xq_bytes), xg_bytes, col_lane, cz, acc)
     int c = 0;
 #pragma unroll 1
