@@ -15,7 +15,7 @@
 //        warp 1   issues tcgen05.mma (M = 128, N = 128, K = 16; A and B from shared-memory descriptors), one fp32
 //                 accumulator of 128 TMEM columns per precision; tcgen05.commit releases a stage;
 //        warps 2-5 epilogue: tcgen05.ld the accumulators, apply alpha / 2^sh / z * sx, store fp32 rows.
-//      No TMA multicast, no clusters.  Every wait on an mbarrier is bounded and reports MATQ_ERR_TIMEOUT.
+//      Every copy goes to the loading CTA only; no clusters.  Every wait on an mbarrier is bounded and reports MATQ_ERR_TIMEOUT.
 #include <cuda.h>
 
 #include "common.cuh"

@@ -31,7 +31,7 @@
 //
 // Data movement.  The CTA's slice of the packed plane is fetched as 128-byte x 128-row boxes of a 2-D tensor map over
 // the plane (uint8, 128-byte swizzle so that 32 rows can be read 16 bytes at a time without bank conflicts; rows and
-// bytes outside the matrix arrive as zeros).  No multicast.  TMEM is allocated before the dependents are released, so
+// bytes outside the matrix arrive as zeros); every copy goes to the loading CTA only.  TMEM is allocated before the dependents are released, so
 // a waiting successor can never starve a predecessor of tensor memory.  Slices of K (grid.y > 1) form a thread-block
 // cluster and are summed through distributed shared memory in rank order.  No global scratch, no atomics.
 #pragma once
