@@ -41,6 +41,28 @@ inline int sm_count() {
     return n;
 }
 
+// Programmatic dependent launch that is safe behind ANY kernel: the launch may begin while the previous kernel of the
+// stream is still running (its start-up then overlaps that kernel's tail), and the kernel calls after_previous_kernel()
+// before its first access to global memory, so it neither reads what the predecessor has not written yet nor writes what
+// it may still read.  let_next_kernel_start() lets a successor launched the same way begin its own start-up early.
+__device__ __forceinline__ void after_previous_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void let_next_kernel_start() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename Kern, typename... Args>
+inline cudaError_t launch_overlapped(Kern kern, dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 // Opts a kernel in, once per device, to the largest dynamic shared memory size an SM offers it (227 KB less the
 // kernel's static shared memory).  The attribute belongs to the function, not to a launch: setting it to each call's
 // size would let two host threads with different shapes undo one another between the setting and the launch.

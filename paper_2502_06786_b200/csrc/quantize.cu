@@ -251,6 +251,8 @@ quantize_rows_reg(const uint16_t* __restrict__ W, int64_t N, int K, int64_t ldw,
                   int32_t* dev_status) {
     __shared__ float s_mn[WARPS], s_mx[WARPS];
     __shared__ int s_bad[WARPS];
+    let_next_kernel_start();
+    after_previous_kernel();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows_per_cta = (WARPS) / wpr;
     const int team = warp / wpr, team_tid = (warp % wpr) * 32 + lane, team_threads = 32 * wpr;
@@ -399,11 +401,11 @@ extern "C" int matq_quantize_clip(const void* W, int64_t N, int64_t K, int64_t l
         if (grid > (int64_t)sms * 32) grid = (int64_t)sms * 32;
 #define MATQ_QUANT_REG(NV) do { \
         if (clip) { \
-            if (warps == 4) quantize_rows_reg<NV, 4, true><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
-            else quantize_rows_reg<NV, 8, true><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            if (warps == 4) launch_overlapped(quantize_rows_reg<NV, 4, true>, dim3((unsigned)grid), dim3(128), 0, s, Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            else launch_overlapped(quantize_rows_reg<NV, 8, true>, dim3((unsigned)grid), dim3(256), 0, s, Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
         } else { \
-            if (warps == 4) quantize_rows_reg<NV, 4, false><<<(unsigned)grid, 128, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
-            else quantize_rows_reg<NV, 8, false><<<(unsigned)grid, 256, 0, s>>>(Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            if (warps == 4) launch_overlapped(quantize_rows_reg<NV, 4, false>, dim3((unsigned)grid), dim3(128), 0, s, Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
+            else launch_overlapped(quantize_rows_reg<NV, 8, false>, dim3((unsigned)grid), dim3(256), 0, s, Wb, N, (int)K, ldw, wpr, gamma, beta, q, alpha, zero, dev_status); \
         } } while (0)
         if (nv <= 2) MATQ_QUANT_REG(2);
         else if (nv <= 3) MATQ_QUANT_REG(3);

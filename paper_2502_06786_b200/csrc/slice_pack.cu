@@ -82,6 +82,8 @@ slice_pack_vec(const uint4* __restrict__ q, int64_t nchunks, int chunks_per_row,
     const int r = PACK_R ? PACK_R : r_runtime;
     const int sh = kCodeBits - r;
     const int64_t stride = (int64_t)gridDim.x * kSliceThreads;
+    let_next_kernel_start();
+    after_previous_kernel();
     for (int64_t i = (int64_t)blockIdx.x * kSliceThreads + threadIdx.x; i < nchunks; i += stride) {
         const uint4 v = ld_stream_u4(q + i);
         if (PACK_R == 2 && !sliced) {
@@ -310,6 +312,9 @@ __device__ __forceinline__ uint32_t chunk_mask(const Sliced& s0, const Sliced& s
 // Sets every flag word to "nothing yet".  The one-pass kernel is launched as its programmatic dependent: it slices,
 // packs and counts while this runs and only waits for it before it touches the first flag.
 __global__ void __launch_bounds__(256) ep_init_flags(uint32_t* __restrict__ row_ptr, int64_t n) {
+    // Launched as a dependent of whatever precedes it: it waits for that kernel FIRST and only then releases
+    // slice_pack_ep, which reads the codes before its own wait (they may be that kernel's output).
+    after_previous_kernel();
     asm volatile("griddepcontrol.launch_dependents;");
     for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) row_ptr[i] = kEpNothing;
 }
@@ -322,6 +327,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
     extern __shared__ __align__(16) uint8_t ep_smem[];
     __shared__ uint32_t base_s, total_s;
     __shared__ int bad_s;
+    let_next_kernel_start();            // every CTA of this grid is resident by now (one wave), so nothing started early can displace one
     const int r = PACK_R ? PACK_R : r_runtime;
     const int sh = kCodeBits - r;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -539,7 +545,7 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     int64_t blocks = (int64_t)sms * per_sm;                   // all resident: the look-back waits rely on it
     if (blocks > ntiles) blocks = ntiles;
     const int64_t init_blocks = (N + 1 + 255) / 256;
-    ep_init_flags<<<(unsigned)(init_blocks < 2 * sms ? init_blocks : 2 * sms), 256, 0, s>>>(reinterpret_cast<uint32_t*>(row_ptr), N + 1);
+    launch_overlapped(ep_init_flags, dim3((unsigned)(init_blocks < 2 * sms ? init_blocks : 2 * sms)), dim3(256), 0, s, reinterpret_cast<uint32_t*>(row_ptr), (int64_t)(N + 1));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3((unsigned)(nwarps * 32));
@@ -567,8 +573,8 @@ void launch_vec(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, 
     int64_t blocks = (nchunks + kSliceThreads - 1) / kSliceThreads;
     const int64_t cap = (int64_t)sm_count() * 32;
     if (blocks > cap) blocks = cap;
-    slice_pack_vec<PACK_R><<<(unsigned)blocks, kSliceThreads, 0, s>>>(
-        reinterpret_cast<const uint4*>(q), nchunks, (int)(K / 16), r, packed, reinterpret_cast<uint4*>(sliced), row_count);
+    launch_overlapped(slice_pack_vec<PACK_R>, dim3((unsigned)blocks), dim3(kSliceThreads), 0, s,
+                      reinterpret_cast<const uint4*>(q), nchunks, (int)(K / 16), r, packed, reinterpret_cast<uint4*>(sliced), row_count);
 }
 
 }  // namespace
