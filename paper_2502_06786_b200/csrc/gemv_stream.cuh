@@ -63,6 +63,7 @@
 #pragma once
 #include <algorithm>
 #include <atomic>
+#include <type_traits>
 
 #include "common.cuh"
 #include "gemv_imma.cuh"
@@ -76,11 +77,12 @@ constexpr int kMaxSlots = 24;
 constexpr int kUnitRow = 1184;                // bytes per row of the largest unit (16 rows)
 constexpr int kMaxTpu = 4;                   // tiles per unit at most
 constexpr int kMaxW = 11;                   // consumer warps at most (with the producer: 12 warps, 168 registers a thread)
+constexpr int kPairs = 1;                    // units of an even number of tiles, two tiles multiplied per pass (see geometry())
 constexpr int kFewW = 8;                    // ... on lists with little work per CTA and for batches: two per sub-partition
 constexpr int kManyItems = 1000;            // items per CTA from which a list gets kMaxW warps: eleven warps measured 1-4 %
                                             // faster on whole decoder stacks and 8-12 % slower on a layer's three matrices
 constexpr int kTileSlots = kMaxW;            // shared-memory accumulators of tiles whose panels are spread over warps
-constexpr int kStaticReserve = 10 * 1024;    // static shared memory of the kernel, rounded up
+constexpr int kStaticReserve = 16 * 1024;    // static shared memory of the kernel, rounded up
 constexpr int kSmallList = 8;
 constexpr int kLargeList = 128;
 constexpr int kSmemLimit = 227 * 1024;
@@ -118,33 +120,43 @@ struct Params {
                               // 2: dependent of ep_rowsum, released after that kernel's own wait (wait before its sums are read)
     int unit_row;             // bytes per row of the largest unit
     int hold;                 // diagnostics: the producer issues no copies, so every wait for a stage runs out
+    int pairs;                // geometry with an even number of tiles per unit (see geometry())
 };
 
-// Shape of a problem's units.  Rows of up to `unit_row` (1184) bytes are staged whole: `tpu` (1 to 4) consecutive tiles are one
-// contiguous run of the plane, rows `row_bytes` apart in shared memory.  Longer rows are cut into `n_panels` panels
-// of `panel_qc` 64-byte chunks (an odd number, so that rows are an odd multiple of 64 bytes apart and the 128-bit
-// loads of a quarter warp fall into different banks; the last panel may be shorter), one tile per unit.
+// Shape of a problem's units.  Short rows are staged whole: `tpu` (1 to 4) consecutive tiles are one contiguous run of the
+// plane, rows `row_bytes` apart in shared memory.  Longer rows are cut into `n_panels` panels of `panel_qc` 64-byte
+// chunks (an odd number, so that rows are an odd multiple of 64 bytes apart and the 128-bit loads of a quarter warp fall
+// into different banks; the last panel may be shorter), and a unit is the box of 16 tpu rows x one panel.
+// `pairs` = 0: rows of up to `unit_row` (1184) bytes are whole, a box is one tile high (panels of up to 17 chunks).
+// `pairs` = 1 (taken at r = 2 only): a unit always holds an even number of tiles, so that two tiles can be multiplied in
+// one pass with one load of the activation fragments: rows of up to unit_row / 2 bytes are whole (2 or 4 tiles), boxes
+// are two tiles high (panels of up to 9 chunks).  The bytes of a unit are the same either way.
 struct Geo {
     int row_bytes, n_qc, tiles, n_panels, panel_qc, stride, contig, tpu;
 };
-__host__ __device__ inline Geo geometry(int N, int K, int r, int unit_row) {
+__host__ __device__ inline Geo geometry(int N, int K, int r, int unit_row, int pairs = 0) {
     const int kUnitBytes = 16 * unit_row;
     Geo g;
     g.row_bytes = K / 8 * r;
     g.n_qc = (g.row_bytes + 63) / 64;
     g.tiles = (N + 15) / 16;
-    if (16 * g.row_bytes <= kUnitBytes) {
+    // Pairs pay at r = 2 only (measured, whole planes: +1 % at K = 2304, +3 % at 3584, +10 % at 9216; at r = 4 and 8 the
+    // narrower panels cost 2-7 % more than the shared fragment loads save).  r = 2 with K % 256 == 128: the half-full
+    // last chunk is handled one tile at a time.
+    if (r != 2 || (g.row_bytes & 63)) pairs = 0;
+    if (16 * (pairs ? 2 : 1) * g.row_bytes <= kUnitBytes) {
         g.contig = 1;
         g.tpu = kUnitBytes / (16 * g.row_bytes);
         if (g.tpu > kMaxTpu) g.tpu = kMaxTpu;
+        if (pairs) g.tpu &= ~1;
         g.n_panels = 1;
         g.panel_qc = g.n_qc;
         g.stride = g.row_bytes;
         return g;
     }
     g.contig = 0;
-    g.tpu = 1;
-    const int max_qc = (kUnitBytes / 16) / 64 - 1;      // 17
+    g.tpu = pairs ? 2 : 1;
+    const int max_qc = pairs ? (kUnitBytes / 32) / 64 : (kUnitBytes / 16) / 64 - 1;      // 9 : 17, both odd
     g.n_panels = (g.n_qc + max_qc - 1) / max_qc;
     g.panel_qc = (g.n_qc + g.n_panels - 1) / g.n_panels;
     g.panel_qc |= 1;
@@ -170,10 +182,10 @@ struct Plan {
 __host__ __device__ inline Plan plan_of(const Geo& g, int T, int W) {
     Plan pl;
     pl.tpu = g.tpu;
-    if (T < W * pl.tpu) pl.tpu = T / W > 1 ? T / W : 1;      // a short share: one tile per unit rather than idle warps
+    if (g.contig && T < W * pl.tpu) pl.tpu = T / W > 1 ? T / W : 1;      // a short share of whole rows: fewer tiles per unit rather than idle warps
     const int Tu = (T + pl.tpu - 1) / pl.tpu;
     pl.split = (Tu < W && g.n_panels > 1) ? 1 : 0;
-    pl.n_units = pl.split ? (T * g.n_panels + W - 1) / W * W : (Tu + W - 1) / W * g.n_panels * W;
+    pl.n_units = pl.split ? (Tu * g.n_panels + W - 1) / W * W : (Tu + W - 1) / W * g.n_panels * W;
     return pl;
 }
 
@@ -235,7 +247,7 @@ __device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, 
     while (p < P.n) {
         const long long i0 = P.p[p].item0;
         if (i0 >= hi) return false;
-        const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r, P.unit_row);
+        const Geo g = geometry(P.p[p].N, P.p[p].K, P.p[p].r, P.unit_row, P.pairs);
         const int tc = tile_cost(g, P.p[p].r);
         const long long a = lo > i0 ? (lo - i0 + tc - 1) / tc : 0;
         const long long b = (hi - i0 + tc - 1) / tc;
@@ -325,46 +337,72 @@ __device__ __forceinline__ void multiply_unit(const unsigned char* wl_p, const u
 #undef MATQ_ITEM
 }
 
-// Two consecutive tiles of a unit at r = 2 in one pass: the B fragments of a chunk (four of the six 128-bit loads of an
-// r = 2 item) are loaded once and used for both tiles' weights.  Tile 0 accumulates in sets 0-3, tile 1 in sets 4-7; a
-// set is used again after eight MMAs.  `wl_p` / `wh_p` belong to tile 0, tile 1 lies `tile_bytes` further.
-__device__ __forceinline__ void multiply_two_tiles_r2(const unsigned char* wl_p, const unsigned char* wh_p, int tile_bytes, uint32_t x_sa, int xq_bytes,
-                                                      int col_lane, const uint4& cz, int n_chunks, int (&acc)[kSets][4]) {
-    uint4 xb[4];
+// Two consecutive tiles of a unit in one pass: the B fragments of a chunk (a third to two thirds of the 128-bit
+// shared-memory loads of an item, and such a load costs a sub-partition more issue time than an MMA) are loaded once
+// and used for both tiles' weights.  Tile 0 accumulates in sets 0-3, tile 1 in sets 4-7; a set is used again after
+// eight MMAs.  `wl_p` / `wh_p` belong to tile 0, tile 1 lies `tile_bytes` further.
+template <int R>
+__device__ __forceinline__ void multiply_two_tiles(const unsigned char* wl_p, const unsigned char* wh_p, int tile_bytes, uint32_t x_sa, int xq_bytes,
+                                                   int col_lane, const uint4& cz, int n_chunks, int (&acc)[kSets][4]) {
+    constexpr int kM2 = (128 / R) / 16;
+    constexpr int kFrag = 2 * kM2;                       // fragments (MMAs per tile) of an item: 2, 4, 8
+    constexpr int kU = kFrag >= 4 ? 1 : 2;               // items per round: at least four fragments, one per set of a tile
+    uint4 xb[kU][kM2];
 #pragma unroll
-    for (int m2 = 0; m2 < 4; ++m2) xb[m2] = cz;
-#pragma unroll 1
-    for (int c = 0; c < n_chunks; ++c) {
-        const uint4 wl0 = *reinterpret_cast<const uint4*>(wl_p + c * 64);
-        const uint4 wh0 = *reinterpret_cast<const uint4*>(wh_p + c * 64);
-        const uint4 wl1 = *reinterpret_cast<const uint4*>(wl_p + tile_bytes + c * 64);
-        const uint4 wh1 = *reinterpret_cast<const uint4*>(wh_p + tile_bytes + c * 64);
+    for (int i = 0; i < kU; ++i)
 #pragma unroll
-        for (int m2 = 0; m2 < 4; ++m2) lds128_if(xb[m2], x_sa + (uint32_t)(c * xq_bytes) + m2 * 256, col_lane);
+        for (int m2 = 0; m2 < kM2; ++m2) xb[i][m2] = cz;
+    auto round = [&](int c, auto n_items) {
+        constexpr int kN = decltype(n_items)::value;
+        uint4 wl[kN][2], wh[kN][2];
 #pragma unroll
-        for (int m2 = 0; m2 < 4; ++m2) {
+        for (int i = 0; i < kN; ++i) {
 #pragma unroll
-            for (int sub = 0; sub < 2; ++sub) {
-                const uint32_t b0 = sub ? xb[m2].z : xb[m2].x, b1 = sub ? xb[m2].w : xb[m2].y;
-#pragma unroll
-                for (int tile = 0; tile < 2; ++tile) {
-                    const uint4& wl = tile ? wl1 : wl0;
-                    const uint4& wh = tile ? wh1 : wh0;
-                    const uint32_t w_lo = m2 == 0 ? wl.x : m2 == 1 ? wl.y : m2 == 2 ? wl.z : wl.w;
-                    const uint32_t w_hi = m2 == 0 ? wh.x : m2 == 1 ? wh.y : m2 == 2 ? wh.z : wh.w;
-                    uint32_t a0, a1, a2, a3;
-                    if (sub == 0) {
-                        a0 = w_lo & 0x03030303u;  a2 = w_lo & 0x0f0f0f0fu;
-                        a1 = w_hi & 0x03030303u;  a3 = w_hi & 0x0f0f0f0fu;
-                    } else {
-                        a0 = w_lo & 0x3f3f3f3fu;  a2 = w_lo;
-                        a1 = w_hi & 0x3f3f3f3fu;  a3 = w_hi;
-                    }
-                    imma::mma_u8u8(acc[4 * tile + (2 * m2 + sub) % 4], a0, a1, a2, a3, b0, b1);
-                }
+            for (int tile = 0; tile < 2; ++tile) {
+                wl[i][tile] = *reinterpret_cast<const uint4*>(wl_p + tile * tile_bytes + (c + i) * 64);
+                wh[i][tile] = *reinterpret_cast<const uint4*>(wh_p + tile * tile_bytes + (c + i) * 64);
             }
+#pragma unroll
+            for (int m2 = 0; m2 < kM2; ++m2) lds128_if(xb[i][m2], x_sa + (uint32_t)((c + i) * xq_bytes) + m2 * 256, col_lane);
         }
-    }
+#pragma unroll
+        for (int i = 0; i < kN; ++i)
+#pragma unroll
+            for (int m2 = 0; m2 < kM2; ++m2)
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub) {
+                    const uint32_t b0 = sub ? xb[i][m2].z : xb[i][m2].x, b1 = sub ? xb[i][m2].w : xb[i][m2].y;
+#pragma unroll
+                    for (int tile = 0; tile < 2; ++tile) {
+                        const uint4& l = wl[i][tile];
+                        const uint4& h = wh[i][tile];
+                        uint32_t a0, a1, a2, a3;
+                        if (R == 8) {
+                            a0 = sub ? l.z : l.x;  a2 = sub ? l.w : l.y;
+                            a1 = sub ? h.z : h.x;  a3 = sub ? h.w : h.y;
+                        } else {
+                            const int j = R == 4 ? 2 * m2 + sub : m2;
+                            const uint32_t w_lo = j == 0 ? l.x : j == 1 ? l.y : j == 2 ? l.z : l.w;
+                            const uint32_t w_hi = j == 0 ? h.x : j == 1 ? h.y : j == 2 ? h.z : h.w;
+                            if (R == 4) {
+                                a0 = w_lo & 0x0f0f0f0fu;  a2 = w_lo;
+                                a1 = w_hi & 0x0f0f0f0fu;  a3 = w_hi;
+                            } else if (sub == 0) {
+                                a0 = w_lo & 0x03030303u;  a2 = w_lo & 0x0f0f0f0fu;
+                                a1 = w_hi & 0x03030303u;  a3 = w_hi & 0x0f0f0f0fu;
+                            } else {
+                                a0 = w_lo & 0x3f3f3f3fu;  a2 = w_lo;
+                                a1 = w_hi & 0x3f3f3f3fu;  a3 = w_hi;
+                            }
+                        }
+                        imma::mma_u8u8(acc[4 * tile + (i * kFrag + 2 * m2 + sub) % 4], a0, a1, a2, a3, b0, b1);
+                    }
+                }
+    };
+    int c = 0;
+#pragma unroll 1
+    for (; c + kU <= n_chunks; c += kU) round(c, std::integral_constant<int, kU>{});
+    if (kU > 1 && c < n_chunks) round(c, std::integral_constant<int, 1>{});
 }
 
 // Activation bytes of one problem in B-fragment order (all chunks of a row).  The byte layout is that of
@@ -690,14 +728,14 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
     int last_it = -1;                                     // latest unit this lane issued a copy for
     while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi)) {
         const Problem& pr = P.p[p - 1];
-        const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row);
+        const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row, P.pairs);
         const int T = t_hi - t_lo;
         const Plan pl = plan_of(G, T, W);
         // Lane l feeds warp l: its units are l, l + W, ...; (tile, panel) and (stage, phase) move by fixed steps.  The
         // lanes advance independently: each probes ITS stage (without suspending) and issues its next copy as soon as
         // its warp has released the stage, so a slow consumer warp never holds back the copies of the others.
         const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
-        int tj = pl.split ? lane / G.n_panels : lane * pl.tpu;
+        int tj = pl.split ? lane / G.n_panels * pl.tpu : lane * pl.tpu;      // first tile of the unit, relative to t_lo
         int pn = pl.split ? lane % G.n_panels : 0;
         int slot = (it0 + lane) % P.slots;
         int use = (it0 + lane) / P.slots;                      // how often the stage has been used before
@@ -726,13 +764,13 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
                     bulk_g2s(dst, pr.packed + row0 * G.row_bytes, bytes, bar);
                     last_it = it0 + s;
                 } else {
-                    mbar_arrive_expect_tx(bar, (uint32_t)(16 * G.stride));     // the whole box, zeros included
+                    mbar_arrive_expect_tx(bar, (uint32_t)(16 * G.tpu * G.stride));     // the whole box, zeros included
                     tensor_g2s(dst, &P.tm[p - 1], pn * G.panel_qc * 8, (t_lo + tj) * 16, bar);
                     last_it = it0 + s;
                 }
                 if (pl.split) {
-                    tj += step_t; pn += step_p;
-                    if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
+                    tj += step_t * pl.tpu; pn += step_p;
+                    if (pn >= G.n_panels) { pn -= G.n_panels; tj += pl.tpu; }
                 } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
                 slot += W;
                 if (slot >= P.slots) { slot -= P.slots; ++use; }
@@ -765,14 +803,14 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
     }
 }
 
-// PAIR2: the variant for lists whose problems are all at r = 2 (it processes two tiles of a unit per pass where it can;
-// the other lists keep the smaller kernel: the extra code costs them 1-2 %).
-template <int NP, bool PAIR2>
+// PAIRS: the variant in which the units of r = 2 problems hold an even number of tiles (geometry with pairs = 1), two of
+// which are multiplied per pass with one load of the activation fragments.
+template <int NP, bool PAIRS>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream(const __grid_constant__ Params<NP> P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxSlots], s_empty[kMaxSlots];
-    __shared__ int s_tile[kTileSlots][16][imma::kCols];       // sums of tiles whose panels are spread over warps
+    __shared__ int s_tile[kTileSlots][2][16][imma::kCols];    // sums of tiles (pairs of tiles) whose panels are spread over warps
     __shared__ int s_tile_cnt[kTileSlots];
     __shared__ uint32_t s_rmax[kMaxW];
     __shared__ float s_rsum[kMaxW];
@@ -791,7 +829,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         mbar_init(smem_u32(&s_empty[tid]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < kTileSlots * 16 * imma::kCols; i += blockDim.x) (&s_tile[0][0][0])[i] = 0;
+    for (int i = tid; i < kTileSlots * 2 * 16 * imma::kCols; i += blockDim.x) (&s_tile[0][0][0][0])[i] = 0;
     if (tid < kTileSlots) s_tile_cnt[tid] = 0;
     __syncthreads();
     if (P.pdl) asm volatile("griddepcontrol.launch_dependents;");
@@ -824,7 +862,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         int xexp = 0;
         while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
             const Problem& pr = P.p[p - 1];
-            G = geometry(pr.N, pr.K, pr.r, P.unit_row);
+            G = geometry(pr.N, pr.K, pr.r, P.unit_row, P.pairs);
             const int R = pr.r;
             const int sh = kCodeBits - R;
             const int T = t_hi - t_lo;
@@ -834,7 +872,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             float sc_first[kMaxTpu];
 #pragma unroll
             for (int k = 0; k < kMaxTpu; ++k) {
-                const int tn = pl.split ? warp / G.n_panels : warp * tpu0 + k;      // split mode: one tile per unit
+                const int tn = pl.split ? warp / G.n_panels * tpu0 : warp * tpu0 + k;      // split mode: the first tile of the warp's first unit
                 const long long row = (long long)(t_lo + tn) * 16 + (lane & 15);
                 sc_first[k] = (k < tpu0 && tn < T && row < pr.N) ? (lane < 16 ? pr.alpha[row] : pr.zero[row]) : 0.f;
             }
@@ -888,11 +926,15 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     multiply_item<2, 0>(wl_p + n_chunks * 64, wh_p + n_chunks * 64, x_sa + (uint32_t)(n_chunks * xq_bytes), col_lane, xt, acc);
                 }
             };
-            // r = 2, whole rows in a stage, no half-full chunk: two tiles of a unit per pass (see multiply_two_tiles_r2)
-            const bool pair_tiles = PAIR2 && R == 2 && G.contig && !half_tail;
-            auto multiply2 = [&](const unsigned char* tile_rows, int (&acc)[kSets][4]) {
+            // two tiles of a unit per pass (see multiply_two_tiles); not with a half-full last chunk
+            const bool pair_tiles = PAIRS && R == 2 && !half_tail;
+            auto multiply2 = [&](const unsigned char* tile_rows, int pn, int (&acc)[kSets][4]) {
+                const int q0 = pn * G.panel_qc, q1 = min(q0 + G.panel_qc, G.n_qc);
                 const unsigned char* base = tile_rows + t * 16;
-                multiply_two_tiles_r2(base + (size_t)g * G.stride, base + (size_t)(g + 8) * G.stride, 16 * G.stride, x_sa0, xq_bytes, col_lane, cz, G.n_qc, acc);
+                const unsigned char* wl_p = base + (size_t)g * G.stride;
+                const unsigned char* wh_p = base + (size_t)(g + 8) * G.stride;
+                const uint32_t x_sa = x_sa0 + (uint32_t)(q0 * xq_bytes);
+                multiply_two_tiles<2>(wl_p, wh_p, 16 * G.stride, x_sa, xq_bytes, col_lane, cz, q1 - q0, acc);
             };
             auto zero_acc = [&](int (&acc)[kSets][4]) {
 #pragma unroll
@@ -954,12 +996,17 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             // split mode: the partial sums of tile `cur` go to its accumulator in shared memory; the warp that brings the
             // last of a tile's contributions finishes it (returns true for that warp, with the sums in acc[0])
             auto flush = [&]() -> bool {
-                fold(acc);
-                const int ts = (split_tiles + cur) % kTileSlots;
-                if (t < 3) {
-                    atomicAdd(&s_tile[ts][g][2 * t], acc[0][0]);
-                    atomicAdd(&s_tile[ts][g + 8][2 * t], acc[0][2]);
-                    if (t < 2) { atomicAdd(&s_tile[ts][g][2 * t + 1], acc[0][1]); atomicAdd(&s_tile[ts][g + 8][2 * t + 1], acc[0][3]); }
+                const bool both = pair_tiles && min(pl.tpu, T - cur) >= 2;      // the unit held two tiles: sums in sets 0-3 and 4-7
+                if (both) fold_two(acc); else fold(acc);
+                const int ts = (split_tiles + cur / pl.tpu) % kTileSlots;
+#pragma unroll
+                for (int tile = 0; tile < 2; ++tile) {
+                    if (tile == 1 && !both) break;
+                    if (t < 3) {
+                        atomicAdd(&s_tile[ts][tile][g][2 * t], acc[4 * tile][0]);
+                        atomicAdd(&s_tile[ts][tile][g + 8][2 * t], acc[4 * tile][2]);
+                        if (t < 2) { atomicAdd(&s_tile[ts][tile][g][2 * t + 1], acc[4 * tile][1]); atomicAdd(&s_tile[ts][tile][g + 8][2 * t + 1], acc[4 * tile][3]); }
+                    }
                 }
                 __threadfence_block();
                 __syncwarp();
@@ -969,22 +1016,30 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 if (prev != contributors - 1) return false;
                 __threadfence_block();                                 // last to arrive: every other contribution is visible
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[0][i] = 0;
-                if (t < 3) {
-                    acc[0][0] = s_tile[ts][g][2 * t];      acc[0][2] = s_tile[ts][g + 8][2 * t];
-                    if (t < 2) { acc[0][1] = s_tile[ts][g][2 * t + 1];  acc[0][3] = s_tile[ts][g + 8][2 * t + 1]; }
+                for (int tile = 0; tile < 2; ++tile) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[4 * tile][i] = 0;
+                    if (tile == 1 && !both) break;
+                    if (t < 3) {
+                        acc[4 * tile][0] = s_tile[ts][tile][g][2 * t];      acc[4 * tile][2] = s_tile[ts][tile][g + 8][2 * t];
+                        if (t < 2) { acc[4 * tile][1] = s_tile[ts][tile][g][2 * t + 1];  acc[4 * tile][3] = s_tile[ts][tile][g + 8][2 * t + 1]; }
+                    }
                 }
                 __syncwarp();
-                if (t < 3) {                                           // leave the slot clean for the tile that reuses it
-                    s_tile[ts][g][2 * t] = 0;  s_tile[ts][g + 8][2 * t] = 0;
-                    if (t < 2) { s_tile[ts][g][2 * t + 1] = 0;  s_tile[ts][g + 8][2 * t + 1] = 0; }
+#pragma unroll
+                for (int tile = 0; tile < 2; ++tile) {                 // leave the slot clean for the tiles that reuse it
+                    if (tile == 1 && !both) break;
+                    if (t < 3) {
+                        s_tile[ts][tile][g][2 * t] = 0;  s_tile[ts][tile][g + 8][2 * t] = 0;
+                        if (t < 2) { s_tile[ts][tile][g][2 * t + 1] = 0;  s_tile[ts][tile][g + 8][2 * t + 1] = 0; }
+                    }
                 }
                 if (lane == 0) s_tile_cnt[ts] = 0;
                 return true;
             };
             // unit s = warp, warp + W, ... without divisions in the loop: (tile, panel) and (stage, phase) move by fixed steps
             const int step_t = pl.split ? W / G.n_panels : 0, step_p = pl.split ? W % G.n_panels : 0;
-            int tj = pl.split ? warp / G.n_panels : warp * pl.tpu;        // first tile of the unit (relative to t_lo)
+            int tj = pl.split ? warp / G.n_panels * pl.tpu : warp * pl.tpu;   // first tile of the unit (relative to t_lo)
             int pn = pl.split ? warp % G.n_panels : 0;                    // its panel
             int slot = (it0 + warp) % P.slots;
             uint32_t parity = (uint32_t)(((it0 + warp) / P.slots) & 1);
@@ -993,6 +1048,10 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 if (ep) await_ep();
                 const float ep_rows = ep ? load_ep(row0) : 0.f;
                 finish_tile(pr.y, pr.N, sh, xexp, xsum, row0, acc[0][0], acc[0][1], acc[0][2], acc[0][3], scales, ep_rows, lane, !*abort_flag);
+                if (pair_tiles && min(pl.tpu, T - cur) >= 2) {             // the second tile of the pair
+                    const float ep2 = ep ? load_ep(row0 + 16) : 0.f;
+                    finish_tile(pr.y, pr.N, sh, xexp, xsum, row0 + 16, acc[4][0], acc[4][1], acc[4][2], acc[4][3], load_scales(row0 + 16), ep2, lane, !*abort_flag);
+                }
             };
             for (int s = warp; s < pl.n_units; s += W) {
                 const int n_tiles = tj < T ? min(pl.tpu, T - tj) : 0;     // 0: an empty unit (padding)
@@ -1025,7 +1084,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                     const bool two = pair_tiles && k + 1 < n_tiles;       // this tile and the next in one pass
                     if (k > 0) zero_acc(acc);
                     if (landed) {
-                        if (two) multiply2(rows + (size_t)k * 16 * G.stride, acc);
+                        if (two) multiply2(rows + (size_t)k * 16 * G.stride, pn, acc);
                         else multiply(rows + (size_t)k * 16 * G.stride, pn, acc);
                     }
                     if (k + (two ? 1 : 0) == n_tiles - 1) {               // the last read of the stage is done
@@ -1044,12 +1103,11 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                         finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[0][0], acc[0][1], acc[0][2], acc[0][3],
                                     k == 0 ? sc[0] : k == 1 ? sc[1] : k == 2 ? sc[2] : sc[3],
                                     k == 0 ? epv[0] : k == 1 ? epv[1] : k == 2 ? epv[2] : epv[3], lane, !*abort_flag);
-                        if (two) {
-                            ++k;
-                            finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k) * 16, acc[4][0], acc[4][1], acc[4][2], acc[4][3],
-                                        k == 1 ? sc[1] : sc[3], k == 1 ? epv[1] : epv[3], lane, !*abort_flag);
-                        }
+                        if (two)
+                            finish_tile(pr.y, pr.N, sh, xexp, xsum, (long long)(t_lo + tj + k + 1) * 16, acc[4][0], acc[4][1], acc[4][2], acc[4][3],
+                                        k == 0 ? sc[1] : sc[3], k == 0 ? epv[1] : epv[3], lane, !*abort_flag);
                     }
+                    if (two) ++k;                                         // the pass covered the next tile too
                 }
                 if (n_tiles == 0) {
                     __syncwarp();
@@ -1057,15 +1115,15 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 }
                 // next unit of this warp
                 if (pl.split) {
-                    tj += step_t; pn += step_p;
-                    if (pn >= G.n_panels) { pn -= G.n_panels; ++tj; }
+                    tj += step_t * pl.tpu; pn += step_p;
+                    if (pn >= G.n_panels) { pn -= G.n_panels; tj += pl.tpu; }
                 } else if (++pn == G.n_panels) { pn = 0; tj += W * pl.tpu; }
                 slot += W;
                 if (slot >= P.slots) { slot -= P.slots; parity ^= 1u; }
             }
             if (pl.split) {
                 if (cur >= 0 && flush()) finish_split((long long)(t_lo + cur) * 16, sc[0]);
-                split_tiles += T;
+                split_tiles += (T + pl.tpu - 1) / pl.tpu;
             }
             it0 += pl.n_units;
         }
@@ -1115,13 +1173,13 @@ inline bool eligible(int64_t N, int64_t K, int r) {
     return warps_for(xs_bytes_of(g, r), slot_bytes_of(g)) >= kMinW;
 }
 
-// Tensor map over a plane as [N][row_bytes / 8] 64-bit words with a box of 16 rows x one panel.
+// Tensor map over a plane as [N][row_bytes / 8] 64-bit words with a box of 16 tpu rows x one panel.
 inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, const Geo& g) {
     t5::EncodeTiledFn fn = t5::encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)(g.row_bytes / 8), (cuuint64_t)N};
     const cuuint64_t strides[1] = {(cuuint64_t)g.row_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)(g.stride / 8), 16u};
+    const cuuint32_t box[2] = {(cuuint32_t)(g.stride / 8), (cuuint32_t)(16 * g.tpu)};
     const cuuint32_t estr[2] = {1u, 1u};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<uint8_t*>(packed), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1132,11 +1190,15 @@ template <int NP>
 inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     static std::atomic<unsigned long long> smem_ok{0}, smem_ok2{0};
     Params<NP> P;
+    // Lists at r = 2 only take the kernel variant with pair units (the others keep the smaller kernel: the extra code
+    // costs them 2-3 %).
+    int pairs = kPairs;
+    for (int i = 0; i < n; ++i) pairs = pairs && (hp[i].N == 0 || hp[i].r == 2);
     long long items = 0, tiles = 0;
     for (int i = 0; i < n; ++i) {
         if (hp[i].N == 0) continue;
         if (!eligible(hp[i].N, hp[i].K, hp[i].r)) return MATQ_ERR_SHAPE;
-        const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
+        const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow, pairs);
         items += (long long)g.tiles * tile_cost(g, hp[i].r);
         tiles += g.tiles;
     }
@@ -1156,7 +1218,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
         q.x = static_cast<const __nv_bfloat16*>(hp[i].x); q.y = hp[i].y;
         q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.B = 1;
         q.item0 = item0;
-        const Geo g = geometry(q.N, q.K, q.r, unit_row);
+        const Geo g = geometry(q.N, q.K, q.r, unit_row, pairs);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
         item0 += (long long)g.tiles * tile_cost(g, q.r);
         xs_bytes = std::max(xs_bytes, xs_bytes_of(g, q.r));
@@ -1209,10 +1271,9 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     }
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
-    bool all_r2 = true;
-    for (int i = 0; i < m; ++i) all_r2 = all_r2 && P.p[i].r == 2;
-    auto kern = all_r2 ? gemv_stream<NP, true> : gemv_stream<NP, false>;
-    if (!opt_in_max_smem(kern, all_r2 ? smem_ok2 : smem_ok)) return MATQ_ERR_CUDA;
+    P.pairs = pairs;
+    auto kern = pairs ? gemv_stream<NP, true> : gemv_stream<NP, false>;
+    if (!opt_in_max_smem(kern, pairs ? smem_ok2 : smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)((W + 1) * 32));

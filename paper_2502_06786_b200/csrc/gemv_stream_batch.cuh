@@ -499,7 +499,7 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
 inline int groups_of(int64_t B) { return B <= 2 ? 1 : B <= 4 ? 2 : 4; }
 
 // static shared memory of the batched kernel with G groups, rounded up
-inline int static_reserve_batch(int G) { return kStaticReserve + (G - 1) * 6 * 1024; }
+inline int static_reserve_batch(int G) { return (10 + (G - 1) * 6) * 1024; }
 
 // Whether a problem with B vectors (2 <= B <= kMaxBatch) can take the batched path.
 inline bool eligible_batch(int64_t N, int64_t K, int r, int64_t B) {
@@ -553,7 +553,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     W = pick_warps(W, fit);
     const int slots = fit / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
-    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = kUnitRow; P.hold = hold ? 1 : 0;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = kUnitRow; P.hold = hold ? 1 : 0; P.pairs = 0;
     auto kern = gemv_stream_batch<NP, G>;
     if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
