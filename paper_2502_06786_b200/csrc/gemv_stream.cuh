@@ -34,6 +34,8 @@
 //       - when the share has at least W tiles, the units are ordered so that a
 //         warp receives all panels of "its" tiles; it keeps the sums in
 //         registers and finishes the 16 outputs alone (three shuffles per row);
+//         at r = 2 a unit holds two tiles and both are multiplied in one pass,
+//         so that the activation fragments are loaded once for 32 rows;
 //       - when it has fewer tiles than warps and rows of several panels, the
 //         panels of a tile are spread over the warps; each adds its partial
 //         sums to a small accumulator in shared memory with integer atomics and

@@ -46,10 +46,12 @@ def _to_device(p, x_dev=None):
 @pytest.mark.parametrize("r", [8, 4, 2])
 @pytest.mark.parametrize("N,K", [(1024, 1024), (300, 2304), (130, 9216), (77, 3584), (3, 128), (257, 14336), (64, 256),
                                  (2304, 9216), (500, 2432), (129, 384), (9216, 2304), (128, 128), (40000, 128),
-                                 (5000, 256), (33, 16384), (33, 32768), (20000, 384), (14336, 3584), (1, 640), (17, 896)])
+                                 (5000, 256), (33, 16384), (33, 32768), (20000, 384), (14336, 3584), (1, 640), (17, 896),
+                                 (37900, 3584)])
 def test_stream_single_problem(r, N, K):
     # every stage shape: 1, 2 and 4 tiles per row block, one and several K panels, half-full last chunks (r = 2,
-    # K % 256 == 128), fewer tiles than SMs and many tiles per SM, the last tile ragged
+    # K % 256 == 128), fewer tiles than SMs and many tiles per SM, the last tile ragged; 37900 x 3584: rows in several
+    # K panels with at least as many pairs of tiles per CTA as warps (two tiles per pass at r = 2, sums kept across panels)
     p = _problem(N, K, r, 500 + N + r)
     status = status_word()
     y = mq.gemv(dev(p["packed"]), K, r, dev(p["a"]), dev(p["z"]), bf16_dev(p["x"]), flags=mq.GEMV_STREAM | mq.GEMV_PDL,
@@ -59,8 +61,9 @@ def test_stream_single_problem(r, N, K):
 
 
 @pytest.mark.parametrize("r", [4, 2])
-@pytest.mark.parametrize("N,K", [(9216, 2304), (2304, 9216), (300, 2432), (2048, 3584), (70, 128)])
+@pytest.mark.parametrize("N,K", [(9216, 2304), (2304, 9216), (300, 2432), (2048, 3584), (70, 128), (4800, 3584), (37900, 3584)])
 def test_stream_extra_precision(r, N, K):
+    # 4800 x 3584: pairs of tiles whose K panels are spread over warps; 37900 x 3584: pairs kept by one warp across panels
     p = _problem(N, K, r, 900 + r, ep=True)
     d = _to_device(p)
     y = mq.gemv(d["packed"], K, r, d["alpha"], d["zero"], d["x"].reshape(1, -1), ovf_row_ptr=d["ovf_row_ptr"],
