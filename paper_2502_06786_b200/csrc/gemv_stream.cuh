@@ -805,9 +805,12 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
     }
 }
 
-// PAIRS: the variant in which the units of r = 2 problems hold an even number of tiles (geometry with pairs = 1), two of
-// which are multiplied per pass with one load of the activation fragments.
-template <int NP, bool PAIRS>
+// RF: 0 = the problems of the list may differ in r; 8, 4, 2 = they are all at that precision, and only that precision's
+// code is compiled into the variant.  The kernel is sensitive to its size (the warps of a CTA are at different places of
+// it, "no instruction" is its most frequent stall): a variant per precision is 3-6 % faster than the one that holds all
+// three.  The r = 2 variant uses pair units (geometry with pairs = 1): two tiles are multiplied per pass with one load
+// of the activation fragments.
+template <int NP, int RF>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream(const __grid_constant__ Params<NP> P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -865,7 +868,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
             const Problem& pr = P.p[p - 1];
             G = geometry(pr.N, pr.K, pr.r, P.unit_row, P.pairs);
-            const int R = pr.r;
+            const int R = RF ? RF : pr.r;
             const int sh = kCodeBits - R;
             const int T = t_hi - t_lo;
             const Plan pl = plan_of(G, T, W);
@@ -929,7 +932,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 }
             };
             // two tiles of a unit per pass (see multiply_two_tiles); not with a half-full last chunk
-            const bool pair_tiles = PAIRS && R == 2 && !half_tail;
+            const bool pair_tiles = RF == 2 && kPairs && !half_tail;
             auto multiply2 = [&](const unsigned char* tile_rows, int pn, int (&acc)[kSets][4]) {
                 const int q0 = pn * G.panel_qc, q1 = min(q0 + G.panel_qc, G.n_qc);
                 const unsigned char* base = tile_rows + t * 16;
@@ -1190,12 +1193,14 @@ inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, co
 
 template <int NP>
 inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
-    static std::atomic<unsigned long long> smem_ok{0}, smem_ok2{0};
+    static std::atomic<unsigned long long> smem_ok[4] = {};
     Params<NP> P;
-    // Lists at r = 2 only take the kernel variant with pair units (the others keep the smaller kernel: the extra code
-    // costs them 2-3 %).
-    int pairs = kPairs;
-    for (int i = 0; i < n; ++i) pairs = pairs && (hp[i].N == 0 || hp[i].r == 2);
+    // the precision the whole list is at (0: mixed) selects the kernel variant; lists at r = 2 get pair units
+    int rf = -1;
+    for (int i = 0; i < n; ++i)
+        if (hp[i].N != 0) rf = rf < 0 ? hp[i].r : (rf == hp[i].r ? rf : 0);
+    if (rf < 0) rf = 0;
+    const int pairs = (rf == 2) ? kPairs : 0;
     long long items = 0, tiles = 0;
     for (int i = 0; i < n; ++i) {
         if (hp[i].N == 0) continue;
@@ -1274,8 +1279,8 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
     P.pairs = pairs;
-    auto kern = pairs ? gemv_stream<NP, true> : gemv_stream<NP, false>;
-    if (!opt_in_max_smem(kern, pairs ? smem_ok2 : smem_ok)) return MATQ_ERR_CUDA;
+    auto kern = rf == 8 ? gemv_stream<NP, 8> : rf == 4 ? gemv_stream<NP, 4> : rf == 2 ? gemv_stream<NP, 2> : gemv_stream<NP, 0>;
+    if (!opt_in_max_smem(kern, smem_ok[rf == 8 ? 3 : rf == 4 ? 2 : rf == 2 ? 1 : 0])) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)((W + 1) * 32));
