@@ -809,8 +809,9 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
 // code is compiled into the variant.  The kernel is sensitive to its size (the warps of a CTA are at different places of
 // it, "no instruction" is its most frequent stall): a variant per precision is 3-6 % faster than the one that holds all
 // three.  The r = 2 variant uses pair units (geometry with pairs = 1): two tiles are multiplied per pass with one load
-// of the activation fragments.
-template <int NP, int RF>
+// of the activation fragments.  LISTS: whether any problem has extra-precision lists (the code that reads ep_rowsum's
+// sums is compiled in only then).
+template <int NP, int RF, bool LISTS>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream(const __grid_constant__ Params<NP> P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -974,7 +975,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             int cur = -1;                                              // split mode: tile whose partial sums are in `acc`
             float sc[kMaxTpu], sc_next[kMaxTpu];
             float epv[kMaxTpu], epv_next[kMaxTpu];                    // extra precision: the sparse term of a tile's rows (lanes 0-15)
-            const bool ep = pr.ovf_row_ptr != nullptr;
+            const bool ep = LISTS && pr.ovf_row_ptr != nullptr;          // LISTS: some problem of the list has extra-precision lists
             // The sparse term is left in y by ep_rowsum (plain coherent loads).  Behind that kernel (pdl == 2) this one
             // starts before the sums are complete: it waits for them when it first needs one, and until then the loads a
             // round ahead are skipped (`epv_ok` / `epv_next_ok`: whether the registers hold loaded values).
@@ -1193,7 +1194,7 @@ inline bool make_plane_map(CUtensorMap* tm, const uint8_t* packed, int64_t N, co
 
 template <int NP>
 inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
-    static std::atomic<unsigned long long> smem_ok[4] = {};
+    static std::atomic<unsigned long long> smem_ok[8] = {};
     Params<NP> P;
     // the precision the whole list is at (0: mixed) selects the kernel variant; lists at r = 2 get pair units
     int rf = -1;
@@ -1279,8 +1280,9 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
     P.pairs = pairs;
-    auto kern = rf == 8 ? gemv_stream<NP, 8> : rf == 4 ? gemv_stream<NP, 4> : rf == 2 ? gemv_stream<NP, 2> : gemv_stream<NP, 0>;
-    if (!opt_in_max_smem(kern, smem_ok[rf == 8 ? 3 : rf == 4 ? 2 : rf == 2 ? 1 : 0])) return MATQ_ERR_CUDA;
+    auto kern = behind_ep ? (rf == 8 ? gemv_stream<NP, 8, true> : rf == 4 ? gemv_stream<NP, 4, true> : rf == 2 ? gemv_stream<NP, 2, true> : gemv_stream<NP, 0, true>)
+                          : (rf == 8 ? gemv_stream<NP, 8, false> : rf == 4 ? gemv_stream<NP, 4, false> : rf == 2 ? gemv_stream<NP, 2, false> : gemv_stream<NP, 0, false>);
+    if (!opt_in_max_smem(kern, smem_ok[(behind_ep ? 4 : 0) + (rf == 8 ? 3 : rf == 4 ? 2 : rf == 2 ? 1 : 0)])) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)((W + 1) * 32));
