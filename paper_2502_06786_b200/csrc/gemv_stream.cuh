@@ -908,7 +908,7 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
                 else if (R == 4) cz = make_uint4(imma::ones_b0<4>(0), imma::ones_b1<4>(0), imma::ones_b0<4>(1), imma::ones_b1<4>(1));
                 else cz = make_uint4(imma::ones_b0<2>(0), imma::ones_b1<2>(0), imma::ones_b0<2>(1), imma::ones_b1<2>(1));
             }
-            const bool half_tail = (G.row_bytes & 63) != 0;          // r = 2, K % 256 == 128: the last chunk is half full
+            const bool half_tail = R == 2 && (G.row_bytes & 63) != 0;   // r = 2, K % 256 == 128: the last chunk is half full
 
             // panel `pn` of the tile whose rows start at `tile_rows` in a stage
             auto multiply = [&](const unsigned char* tile_rows, int pn, int (&acc)[kSets][4]) {
