@@ -328,6 +328,18 @@ int matq_gemm_multi_static(int src_kind, const void *Wsrc, int64_t N, int64_t K,
                            const int *rs, int n_r, float *const *Y, int64_t ldy,
                            int32_t *dev_status, void *stream);
 
+/*
+ * Testing hook for the error path of the dense forward (matq_gemm_multi, matq_gemm_multi_loss,
+ * matq_gemm_multi_static).  While `on` is non-zero, the tensor-core kernel of every such call issues none of its copies,
+ * and its waits give up after about a millisecond instead of about two seconds (every wait of that kernel is bounded in
+ * SM clock cycles).  Such a call returns MATQ_OK, reports MATQ_ERR_TIMEOUT through dev_status, stores nothing to Y
+ * (loss mode: the loss it writes is meaningless) and frees its tensor memory; alpha, zero and the workspace are written
+ * as usual.  The setting is process-wide and is read when a call is made: do not change it while another thread is
+ * inside one of these calls.  Returns the previous setting.  No copy is in flight when such a kernel exits, and the next
+ * call with the hook off works as usual.
+ */
+int matq_gemm_multi_test_stall(int on);
+
 #ifdef __cplusplus
 }
 #endif

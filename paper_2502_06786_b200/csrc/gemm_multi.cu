@@ -28,7 +28,8 @@ constexpr int kThreads = 192;
 constexpr int kMaxR = 3;
 constexpr int kMaxStages = 8;
 constexpr int kTileBytes = kBM * kBK * 2;          // 16 KB: one 128 x 64 bf16 box
-constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr long long kWaitCycles = 4000000000ll;     // SM clock cycles after which a wait on an mbarrier gives up: about two seconds
+constexpr long long kStallWaitCycles = 2000000ll;   // the same under matq_gemm_multi_test_stall: about a millisecond
 
 struct Params {
     const float* alpha;
@@ -44,15 +45,25 @@ struct Params {
     float* loss_part;     // loss mode: [CTAs][kMaxR] sums of squared errors
     int teacher[kMaxR];   // loss mode, per precision: -1 target only, j another precision's output as the target, 256 + j both
     int32_t* dev_status;
+    long long wait_cycles;   // limit of every wait on an mbarrier
+    int hold;                // tests of the error path: the producer issues no copies
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded in SM clock cycles (the clock is read once per 64 polls; the first reading starts the count).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
     uint32_t done = 0;
-    for (uint32_t it = 0; it < kSpinLimit && !done; ++it)
+    long long t0 = 0;
+    for (uint32_t it = 0; !done; ++it) {
         asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (!done && (it & 63u) == 63u) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit) break;
+        }
+    }
     return done != 0;
 }
 
@@ -127,10 +138,10 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // ---------------- TMA producer
         if (lane == 0) {
             const CUtensorMap* tmb[kMaxR] = {&tm_b0, &tm_b1, &tm_b2};
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kb = 0; kb < nkb && !P.hold; ++kb) {
                 const int s = kb % P.stages;
                 const uint32_t ph = (uint32_t)(kb / P.stages) & 1u;
-                if (!mbar_wait(smem_u32(&s_empty[s]), ph ^ 1u)) { s_timeout = 1; break; }
+                if (!mbar_wait(smem_u32(&s_empty[s]), ph ^ 1u, P.wait_cycles)) { s_timeout = 1; break; }
                 const uint32_t bar = smem_u32(&s_full[s]);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(stage_bytes) : "memory");
                 unsigned char* st = ring + (size_t)s * stage_bytes;
@@ -150,7 +161,12 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             for (int kb = 0; kb < nkb && ok; ++kb) {
                 const int s = kb % P.stages;
                 const uint32_t ph = (uint32_t)(kb / P.stages) & 1u;
-                if (!mbar_wait(smem_u32(&s_full[s]), ph)) { s_timeout = 1; ok = false; break; }
+                if (!mbar_wait(smem_u32(&s_full[s]), ph, P.wait_cycles)) {
+                    s_timeout = 1;                            // visible to the epilogue before the arrival below
+                    __threadfence_block();
+                    ok = false;
+                    break;
+                }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_base = smem_u32(ring + (size_t)s * stage_bytes);
 #pragma unroll
@@ -177,7 +193,8 @@ gemm_multi_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const int quad = warp & 3;
         const int64_t m = m0 + quad * 32 + lane;
         // whole warps agree on the outcome: the reads of tensor memory below are warp-wide
-        const bool done = __all_sync(0xffffffffu, mbar_wait(smem_u32(&s_acc), 0));
+        // (the arrival also comes when the MMA warp gave up: the accumulators are then incomplete and are not used)
+        const bool done = __all_sync(0xffffffffu, mbar_wait(smem_u32(&s_acc), 0, P.wait_cycles)) && *(volatile int*)&s_timeout == 0;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (!done) s_timeout = 1;                           // gave up: report it, read and store nothing
         const float sx = (m < P.M) ? P.sx[m] : 0.f;
@@ -477,6 +494,11 @@ inline int64_t cta_count(int64_t M, int64_t N, int n_r) {
 }  // namespace gm
 }  // namespace matq
 
+// Tests of the error path (matq_gemm_multi_test_stall): process-wide, read when a call builds its launch.
+static std::atomic<int> g_test_stall{0};
+
+extern "C" int matq_gemm_multi_test_stall(int on) { return g_test_stall.exchange(on ? 1 : 0); }
+
 // The forward (Y != NULL, Yt == NULL) or the loss (Yt != NULL, loss_part != NULL; nothing is stored to Y).
 static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K, int c,
                            float* alpha, float* zero, int extra_precision,
@@ -572,6 +594,8 @@ static int gemm_multi_impl(int src_kind, const void* Wsrc, int64_t N, int64_t K,
     for (int i = 0; i < kMaxR; ++i) P.teacher[i] = (teacher && i < n_r) ? teacher[i] : -1;
     P.M = M; P.N = N; P.K = K; P.ldy = ldy; P.n_r = n_r;
     P.dev_status = dev_status;
+    P.hold = g_test_stall.load(std::memory_order_relaxed) ? 1 : 0;
+    P.wait_cycles = P.hold ? kStallWaitCycles : kWaitCycles;
     // A single plane would leave every MMA at N = 128 (shared-memory bound); the CTA then takes 256 channels as two
     // adjacent tiles of the same plane so that one N = 256 instruction covers them.
     P.wide = (n_r == 1 && N > kBN) ? 1 : 0;

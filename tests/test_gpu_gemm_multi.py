@@ -174,6 +174,34 @@ def test_matches_decode_gemv_and_full_path():
         assert np.abs(host(y) - host(Ys[i])).max() <= 1e-3 * rms(host(y))
 
 
+def test_a_wait_that_runs_out_is_a_status_not_a_hang():
+    # matq_gemm_multi_test_stall: the tensor-core kernel issues none of its copies, so the MMA warp's wait for its first
+    # stage and the epilogue's wait for the accumulators run out (bounded in clock cycles).  The kernel must return,
+    # report MATQ_ERR_TIMEOUT, store nothing and free its tensor memory; the same context must then serve the same call.
+    M, N, K = 200, 264, 256
+    W = synth.normal_bf16((N, K), 0.02, 90)
+    st, q, a, z = ref.quantize(W)
+    X = synth.normal_bf16((M, K), 1.0, 91)
+    st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, q, K, X, alpha=a, zero=z)
+    status = status_word()
+    Ys = [torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda") for _ in range(3)]
+    assert mq.gemm_multi_test_stall(True) == 0
+    try:
+        mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(8, 4, 2), alpha=dev(a), zero=dev(z), Ys=Ys, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        assert mq.gemm_multi_test_stall(False) == 1
+    assert int(host(status)[0]) == mq.ERR_TIMEOUT
+    for y in Ys:
+        assert bool(torch.isnan(y).all())               # nothing was stored
+    # tensor memory was given back (a CTA that kept its columns would block the next one on its SM)
+    status.zero_()
+    for _ in range(3):
+        Ys2, _, _ = mq.gemm_multi(mq.SRC_CODES8, dev(q), K, bf16_dev(X), rs=(8, 4, 2), alpha=dev(a), zero=dev(z), dev_status=status)
+        _check(Ys2, Yr)
+    assert int(host(status)[0]) == mq.OK
+
+
 def test_argument_errors_and_empty():
     lib = mq._lib
     fake = C.c_void_p(0x1000)
