@@ -340,6 +340,17 @@ int matq_gemm_multi_static(int src_kind, const void *Wsrc, int64_t N, int64_t K,
  */
 int matq_gemm_multi_test_stall(int on);
 
+/*
+ * Testing hook for the one device-side wait of matq_slice_pack / matq_slice_pack_nested with extra_precision: the
+ * look-back of the one-pass kernel, in which a tile of rows waits for the overflow counts of the tiles before it.  While
+ * `on` is non-zero, the first tile never publishes its count and a look-back gives up after 2^8 polls instead of 2^20;
+ * every later tile then meets "nothing yet" until its limit, or the mark of a tile that has already given up.  Such a
+ * call returns MATQ_OK and reports MATQ_ERR_TIMEOUT through dev_status; the planes are complete, ovf_row_ptr, ovf_col and
+ * ovf_count are not.  Process-wide like the hook above; returns the previous setting.  Shapes that the one-pass kernel
+ * does not take (K % 16 != 0, K > 16384, 2^31 codes or more) have no device-side wait and ignore it.
+ */
+int matq_slice_pack_test_stall(int on);
+
 #ifdef __cplusplus
 }
 #endif

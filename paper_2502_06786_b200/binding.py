@@ -27,7 +27,7 @@ EXPORTS = ["matq_status_string", "matq_version", "matq_packed_row_bytes", "matq_
            "matq_slice_pack", "matq_slice_pack_nested", "matq_gemv_workspace_bytes", "matq_gemv", "matq_gemv_grouped", "matq_gemv_grouped_launches",
            "matq_gemm_multi_workspace_bytes", "matq_gemm_multi",
            "matq_gemm_multi_loss_workspace_bytes", "matq_gemm_multi_loss",
-           "matq_gemm_multi_test_stall",
+           "matq_gemm_multi_test_stall", "matq_slice_pack_test_stall",
            "matq_gemm_multi_static_max_bytes", "matq_gemm_multi_static"]
 
 
@@ -84,6 +84,8 @@ def _load():
                                          C.POINTER(C.c_int), i32, C.POINTER(C.c_float), C.POINTER(C.c_int), vp, i64, vp, vp, sz, vp, vp]
     lib.matq_gemm_multi_test_stall.restype = i32
     lib.matq_gemm_multi_test_stall.argtypes = [i32]
+    lib.matq_slice_pack_test_stall.restype = i32
+    lib.matq_slice_pack_test_stall.argtypes = [i32]
     lib.matq_gemm_multi_static_max_bytes.restype = sz
     lib.matq_gemm_multi_static_max_bytes.argtypes = []
     lib.matq_gemm_multi_static.restype = i32
@@ -361,6 +363,11 @@ def gemm_multi_loss(src_kind, Wsrc, K, X, Yt, lambdas, rs=(8, 4, 2), alpha=None,
                                    workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream())
     _check(st, "matq_gemm_multi_loss")
     return loss, alpha, zero
+
+
+def slice_pack_test_stall(on) -> int:
+    """matq_slice_pack_test_stall: switch the one-pass slice kernel's "first tile never publishes" test mode."""
+    return int(_lib.matq_slice_pack_test_stall(1 if on else 0))
 
 
 def gemm_multi_test_stall(on) -> int:

@@ -291,6 +291,7 @@ ovf_fill_batched(const uint8_t* __restrict__ q, int64_t N, int64_t K, int r, con
 // poisons the flags after it and reports MATQ_ERR_TIMEOUT instead of hanging.
 constexpr uint32_t kEpNothing = 0xffffffffu, kEpPartial = 0x80000000u, kEpPoison = 0xc0000000u;
 constexpr int kEpSpinLimit = 1 << 20;
+constexpr int kEpStallSpinLimit = 1 << 8;    // under matq_slice_pack_test_stall
 constexpr int kEpWindows = 4;              // look-back windows of 32 tiles fetched per round trip
 constexpr size_t kEpSmemLimit = 160 * 1024;
 constexpr int kEpBatch = 6;                // 16-byte loads a lane has in flight
@@ -323,7 +324,10 @@ template <int PACK_R>
 __global__ void __launch_bounds__(1024)
 slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, int rows_per_warp,
               uint8_t* __restrict__ packed, uint8_t* __restrict__ packed4, uint8_t* __restrict__ sliced, uint32_t* __restrict__ row_ptr,
-              uint16_t* __restrict__ ovf_col, int64_t capacity, int64_t* __restrict__ total_out, int32_t* dev_status) {
+              uint16_t* __restrict__ ovf_col, int64_t capacity, int64_t* __restrict__ total_out, int32_t* dev_status,
+              int spin_limit, int hold) {
+    // spin_limit: polls of a look-back before it gives up.  hold (tests of that path): the first tile never publishes
+    // its prefix, so every later tile's look-back meets "nothing yet" until its limit, or the poison of a tile before it.
     extern __shared__ __align__(16) uint8_t ep_smem[];
     __shared__ uint32_t base_s, total_s;
     __shared__ int bad_s;
@@ -425,7 +429,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
                             nothing |= f[w] == kEpNothing;
                         }
                         if (!__any_sync(0xffffffffu, nothing)) break;
-                        if (++spins > kEpSpinLimit) { bad = true; break; }
+                        if (++spins > spin_limit) { bad = true; break; }
                         __nanosleep(40);
                     }
                     if (bad) break;
@@ -449,7 +453,7 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
                     st_flag(row_ptr + last_row + 1, kEpPoison);
                     report(dev_status, MATQ_ERR_TIMEOUT);
                     if (t == ntiles - 1) *total_out = 0;
-                } else {
+                } else if (!(hold && t == 0)) {
                     st_flag(row_ptr + last_row + 1, base + tile_total);   // the thread that wrote the partial replaces it
                     if (t == 0) row_ptr[0] = 0;
                     if (t == ntiles - 1) {
@@ -516,6 +520,9 @@ slice_pack_ep(const uint8_t* __restrict__ q, int64_t N, int K, int r_runtime, in
     }
 }
 
+// Tests of the look-back's give-up path (matq_slice_pack_test_stall): process-wide, read when a call builds its launch.
+static std::atomic<int> g_test_stall{0};
+
 // Returns MATQ_ERR_SHAPE when no tile fits the shared-memory budget (the caller then uses the three-kernel chain).
 template <int PACK_R>
 int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, uint8_t* sliced, int32_t* row_ptr,
@@ -558,8 +565,9 @@ int launch_ep(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, ui
     cfg.numAttrs = 1;
     const int K32 = (int)K;
     uint32_t* flags = reinterpret_cast<uint32_t*>(row_ptr);
+    const int hold = g_test_stall.load(std::memory_order_relaxed) ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, slice_pack_ep<PACK_R>, q, N, K32, r, rpw, packed, packed4, sliced, flags, ovf_col, capacity, total,
-                           dev_status) != cudaSuccess) {
+                           dev_status, hold ? kEpStallSpinLimit : kEpSpinLimit, hold) != cudaSuccess) {
         cudaGetLastError();
         return MATQ_ERR_CUDA;
     }
@@ -579,6 +587,8 @@ void launch_vec(const uint8_t* q, int64_t N, int64_t K, int r, uint8_t* packed, 
 
 }  // namespace
 }  // namespace matq
+
+extern "C" int matq_slice_pack_test_stall(int on) { return matq::g_test_stall.exchange(on ? 1 : 0); }
 
 extern "C" int64_t matq_packed_row_bytes(int64_t K, int r) {
     if (!(r == 8 || r == 4 || r == 2) || K <= 0 || (K % (8 / r)) != 0) return -1;

@@ -255,6 +255,37 @@ def test_extra_precision_capacity_error_is_a_status():
     assert int(host(cnt)[0]) == 0
 
 
+@pytest.mark.parametrize("nested", [False, True])
+def test_a_look_back_that_runs_out_is_a_status_not_a_hang(nested):
+    # matq_slice_pack_test_stall: the first tile of the one-pass kernel never publishes its overflow count, so the
+    # look-back of every later tile meets "nothing yet" until its (shortened) limit or the mark of a tile that gave up.
+    # The call must return, report MATQ_ERR_TIMEOUT and still write the planes; the next call must be bit-exact.
+    N, K = 9216, 2304
+    q = synth.skewed_codes((N, K), 0.005, 224, 1234)
+    want2 = ref.slice_pack(q, 2, extra_precision=True)
+    qd = dev(q)
+    status = status_word()
+    call = (lambda: mq.slice_pack_nested(qd, extra_precision=True, dev_status=status)) if nested else \
+           (lambda: mq.slice_pack(qd, 2, extra_precision=True, dev_status=status))
+    assert mq.slice_pack_test_stall(True) == 0
+    try:
+        out = call()
+        torch.cuda.synchronize()
+    finally:
+        assert mq.slice_pack_test_stall(False) == 1
+    assert int(host(status)[0]) == mq.ERR_TIMEOUT
+    assert np.array_equal(host(out["packed2" if nested else "packed"]), want2["packed"])      # the planes do not wait for anything
+    if nested:
+        assert np.array_equal(host(out["packed4"]), ref.slice_pack(q, 4)["packed"])
+    status.zero_()
+    out = call()
+    cnt = int(host(out["ovf_count"])[0])
+    assert cnt == want2["ovf_count"]
+    assert np.array_equal(host(out["ovf_row_ptr"]), want2["ovf_row_ptr"])
+    assert np.array_equal(host(out["ovf_col"])[:cnt], want2["ovf_col"])
+    assert int(host(status)[0]) == mq.OK
+
+
 # ---------------------------------------------------------------------- gemv
 
 def _gemv_case(N, K, B, r, seed, ep=False, flags=0):
