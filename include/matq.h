@@ -144,6 +144,8 @@ int matq_quantize_clip(const void *W, int64_t N, int64_t K, int64_t ldw, int c,
  *   packed           out  uint8 [N, K*r/8]; NULL allowed (then only the other outputs are written);
  *                         non-NULL requires r in {8, 4, 2} and K % (8/r) == 0
  *   sliced_unpacked  out  uint8 [N, K] = S(q, r) of Eq. 6, any 1 <= r <= 8; NULL allowed
+ *                         (an interpolated precision such as r = 6 or 3, Section 5.1, is served in decode by passing
+ *                         this array to matq_gemv as an r = 8 plane: dequantisation is alpha * (S - z) either way)
  *   Extra precision (Eq. 8 keeps bucket 2^r): the plane holds the CLAMPED field,
  *   so it is byte-identical to the standard plane, and the elements whose Eq. 8
  *   value is one bucket higher (exactly those with q >= 2^c - 2^(sh-1)) are listed:

@@ -466,6 +466,29 @@ def test_gemv_strided_x_and_y():
     assert np.all(host(yw)[:, N:] == -1.0)
 
 
+@pytest.mark.parametrize("r", [7, 6, 5, 3, 1])
+def test_interpolated_precisions_decode_from_an_unpacked_slice(r):
+    # Section 5.1 serves precisions that were not trained (int6, int3, ...) by slicing the same int8 codes.  For decode the
+    # slice S(q, r) of Eq. 6, one byte per weight, IS an 8-bit plane: y = sum_k x alpha (S - z) is the r = 8 GEMV on it.
+    # Checked against the oracle's dequantised product at that r (a different oracle routine than its GEMV).
+    N, K = 520, 2304
+    W = synth.normal_bf16((N, K), 0.02, 950 + r)
+    st, q, a, z = ref.quantize(W)
+    sl = mq.slice_pack(dev(q), r, want_packed=False, want_unpacked=True)["sliced"]
+    st, S = ref.slice_values(q, r)
+    assert st == ref.OK and np.array_equal(host(sl), S.astype(np.uint8))
+    for B, tol in ((1, TOL_INT8), (4, TOL_TENSOR)):
+        x = synth.normal_bf16((B, K), 1.0, 960 + r + B)
+        st, Yr, _, _ = ref.gemm_multi(ref.SRC_CODES8, q, K, x, rs=(r,), alpha=a, zero=z)
+        assert st == ref.OK
+        y = mq.gemv(sl, K, 8, dev(a), dev(z), bf16_dev(x))
+        assert np.abs(host(y).reshape(B, N) - Yr[0]).max() <= tol * rms(Yr[0])
+        yg = torch.empty((B, N), dtype=torch.float32, device="cuda")
+        ad, zd, xd = dev(a), dev(z), bf16_dev(x)
+        mq.gemv_grouped(mq.gemv_group([dict(packed=sl, K=K, r=8, alpha=ad, zero=zd, x=xd, y=yg)]))
+        assert np.abs(host(yg) - Yr[0]).max() <= TOL_INT8 * rms(Yr[0])
+
+
 def test_full_path_quantize_slice_pack_gemv():
     # bf16 weights -> codes -> plane -> y, everything on the GPU, against the oracle end to end.
     N, K, B = 260, 2304, 2
