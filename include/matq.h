@@ -217,21 +217,27 @@ int matq_gemv(const uint8_t *packed, int64_t N, int64_t K, int c, int r,
  *      an x_j of the same call).  With one vector per problem (B <= 1) the results are those of matq_gemv's integer
  *      path (exact integer sums, reproducible: a problem gives the same bits alone, in any list and however the list
  *      is split over CTAs).
- *      Batches (2 <= B <= 16, no lists): the plane is read from HBM once for up to 8 vectors.  The sums are exact
- *      integers again, but an activation is a 22-bit integer relative to the largest magnitude of ITS vector, and a
- *      field that sits s bits up in its byte meets its activation divided by 2^s: the rounding step is 2^-22 (r = 8),
- *      2^-18 (r = 4), 2^-16 (r = 2) of twice the vector's largest magnitude (about 1e-6, 2e-5, 6e-5 of rms(y) for
- *      Gaussian activations).  A vector whose largest element is thousands of times its typical one loses
- *      accordingly; such vectors belong in problems of their own (B = 1: 30-bit activations) or in matq_gemv's
- *      default path (bf16 products).  A batch that does not fit one launch's shared memory (more than 8 vectors;
- *      more than 4 at K = 9216) is cut into problems that share the plane; r = 2 batches need K % 256 == 0.
+ *      Batches (2 <= B <= 16, no lists): the plane is read from HBM once for up to 16 vectors (8 at r = 2).  The
+ *      sums are exact integers again; what is rounded is the activation, relative to the largest magnitude of ITS
+ *      vector.  B = 2, and every batch at r = 2: a 22-bit integer, and a field that sits s bits up in its byte meets its
+ *      activation divided by 2^s, so the rounding step is 2^-22 (r = 8), 2^-18 (r = 4), 2^-16 (r = 2) of twice the
+ *      vector's largest magnitude (about 1e-6, 2e-5, 6e-5 of rms(y) for Gaussian activations).  B >= 3 at r = 8 and
+ *      r = 4: a 15-bit integer and its sign (two signed base-256 digits, four vectors per 8-column MMA instead of
+ *      two), a rounding step of 2^-14 of the power of two at or below the vector's largest magnitude (2^-13 when that
+ *      magnitude's bf16 significand is all ones), the same for both fields: about 4e-5 of rms(y) for Gaussian
+ *      activations, below what the 8-bit significands of the bf16 inputs themselves resolve, and well inside the
+ *      1e-2 rms(y) of the tensor-core paths.  In either form a vector whose largest element is thousands of times its
+ *      typical one loses accordingly; such vectors belong in problems of their own (B = 1: 30-bit activations) or in
+ *      matq_gemv's default path (bf16 products).  A batch that does not fit one launch's shared memory (at K = 9216:
+ *      more than 4 vectors) is cut into problems that share the plane; r = 2 batches need K % 256 == 0.
  *   problems   in   HOST array of n_problems descriptors; the pointers inside are DEVICE pointers:
  *                     packed uint8 [N, K*r/8] 16-byte aligned, alpha / zero fp32 [N], ovf_row_ptr / ovf_col both NULL
  *                     or both given (B <= 1 only), x bf16 [K] (or [B, K], rows K apart) 16-byte aligned, y fp32 [N]
  *                     (or [B, N], rows N apart).  r in {8, 4, 2}, K % 128 == 0, K <= 32768.
  *                     A problem with N == 0 is skipped.  The array is read during the call only.
  *   n_problems      any number >= 0; up to 128 problems share a launch, longer lists take several; single vectors
- *                   and batches of 2, 3-4 and 5-8 vectors go to launches of their own
+ *                   and batches that need 1, 2 or 4 column groups (of two or of four vectors) go to launches of
+ *                   their own
  *   flags           0 or MATQ_GEMV_PDL (MATQ_GEMV_TEST_STALL for tests of the error path; meaning of PDL as for matq_gemv: no plane, alpha, zero or list of the call is
  *                   written by the previous kernel of the stream)
  *   A wait inside the kernel that does not end within about two seconds sets dev_status = MATQ_ERR_TIMEOUT; the

@@ -38,11 +38,14 @@ namespace gstream {
 constexpr int kP2 = 21;                      // batched activations become integers below 2^(kP2 + 1)
 constexpr int kPairCols = 7;                 // columns of a group: 3 + 3 bytes and the constant column
 constexpr int kPairUnit = (kPairCols - 1) * 64;   // bytes of a staged (chunk, unit) block: the six byte columns (the constant column lives in registers)
-constexpr int kMaxBatch = 8;
+constexpr int kMaxBatch = 8;                 // vectors of a problem in pair groups (4 groups of 2)
+constexpr int kP4 = 14;                      // quad groups: activations become integers of magnitude below 2^(kP4 + 1)
+constexpr int kQuadUnit = 8 * 64;            // bytes of a staged (chunk, unit) block of a quad group: two signed digits of four vectors
+constexpr int kMaxVec = 16;                  // vectors of a problem in quad groups (4 groups of 4)
 constexpr int kWideFit = 7;                  // stages a problem's own shapes must leave room for to share a launch with the short rows
 
 // Staged bytes of one group for a problem (all chunks of a row).
-inline size_t xs_group_bytes_of(const Geo& g, int r) { return (size_t)g.n_qc * ((128 / r) / 16) * kPairUnit; }
+inline size_t xs_group_bytes_of(const Geo& g, int r, bool quad = false) { return (size_t)g.n_qc * ((128 / r) / 16) * (quad ? kQuadUnit : kPairUnit); }
 
 // Converts 16 consecutive activations of the two vectors of a group and stores their byte units: column blocks 0-2
 // (first vector) and 3-5 (second).  `dst` points at this item's 16 bytes of column block 0.
@@ -275,17 +278,218 @@ __device__ __noinline__ void finish_tile_pair(float* __restrict__ ya, float* __r
     }
 }
 
-template <int NP, int G>
+
+// ---------------------------------------------------------------------------------------------------------------
+// Quad groups (r = 8 and r = 4, three or more vectors): the eight B columns of a group are TWO SIGNED digits (base 256,
+// each in [-128, 127]) of FOUR vectors; the MMA is u8 x s8, there is no offset and no constant column, and column
+// 2v + d of the result is digit d of vector v's sum, so thread (g, t) of the accumulator fragment holds both digits of
+// vector t for its two rows.  Half the MMAs and B-fragment loads of pair groups for the same vectors.  An activation
+// is rounded to an integer of magnitude at most 2^15 - 256 (15 bits and the sign: 2^-14 of the power of two at or
+// below the vector's largest magnitude, one bit less when that magnitude's significand is all ones).  At r = 4 the
+// upper field is shifted down instead of being left in place, so both fields meet activations of the same scale.
+
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// 16 consecutive activations of one vector as two signed digits: `dst` points at this item's 16 bytes of the vector's
+// low-digit column block, the high-digit block follows it.
+template <int R>
+__device__ __forceinline__ void stage_item_quad(const uint32_t (&raw)[8], float mult, uint4* dst) {
+    uint32_t u[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const uint32_t w = raw[i >> 1];
+        const int V = __float2int_rn(((i & 1) ? bf_hi(w) : bf_lo(w)) * mult);
+        u[i] = (uint32_t)(V + ((V & 0x80) << 1));             // low byte as a signed digit: the high byte takes the carry
+    }
+    uint32_t col[2][4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const uint32_t e0 = u[imma::unit_src<R>(4 * w)], e1 = u[imma::unit_src<R>(4 * w + 1)];
+        const uint32_t e2 = u[imma::unit_src<R>(4 * w + 2)], e3 = u[imma::unit_src<R>(4 * w + 3)];
+        const uint32_t t0 = __byte_perm(e0, e1, 0x5140), t1 = __byte_perm(e2, e3, 0x5140);
+        col[0][w] = __byte_perm(t0, t1, 0x5410);  col[1][w] = __byte_perm(t0, t1, 0x7632);
+    }
+    dst[0] = make_uint4(col[0][0], col[0][1], col[0][2], col[0][3]);
+    dst[4] = make_uint4(col[1][0], col[1][1], col[1][2], col[1][3]);
+}
+
+// As stage_activations_pair, for G groups of four vectors.
+template <int R, int G>
+__device__ __forceinline__ void stage_activations_quad(const __nv_bfloat16* x, int K, int B, int n_qc, unsigned char* xs, size_t group_bytes,
+                                                       int ctid, int nthr, int W, uint32_t (*s_cmax)[kMaxVec], float (*s_csum)[kMaxVec],
+                                                       int* s_xexp, float* s_xsum) {
+    constexpr int kWpp = 128 / R;
+    constexpr int kM2 = kWpp / 16;
+    const int lane = ctid & 31, warp = ctid >> 5;
+    const int n_items = n_qc * kM2 * 4;
+    auto k0_of = [&](int it) {
+        const int tt = it & 3, qm = it >> 2;
+        return ((qm / kM2) * 4 + tt) * kWpp + (qm % kM2) * 16;
+    };
+    for (int c = 0; c < 4 * G; ++c) {
+        uint32_t xmax = 0;
+        float xsum = 0.f;
+        if (c < B) {
+            const __nv_bfloat16* xc = x + (size_t)c * K;
+            for (int it = ctid; it < n_items; it += nthr) {
+                const int k0 = k0_of(it);
+                if (k0 >= K) continue;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint4 v = ld_x4(xc + k0 + 8 * h);
+                    xmax = __vmaxu2(xmax, v.x & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.y & 0x7fff7fffu);
+                    xmax = __vmaxu2(xmax, v.z & 0x7fff7fffu); xmax = __vmaxu2(xmax, v.w & 0x7fff7fffu);
+                }
+            }
+            if (ctid < kSumThreads)                                // fixed order: see stage_activations
+                for (int it = ctid; it < n_items; it += kSumThreads) {
+                    const int k0 = k0_of(it);
+                    if (k0 >= K) continue;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint4 v = ld_x4(xc + k0 + 8 * h);
+                        xsum += ((bf_lo(v.x) + bf_hi(v.x)) + (bf_lo(v.y) + bf_hi(v.y))) + ((bf_lo(v.z) + bf_hi(v.z)) + (bf_lo(v.w) + bf_hi(v.w)));
+                    }
+                }
+        }
+        xmax = max(xmax & 0xffffu, xmax >> 16);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            xmax = max(xmax, __shfl_xor_sync(0xffffffffu, xmax, o));
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, o);
+        }
+        if (lane == 0) { s_cmax[warp][c] = xmax; s_csum[warp][c] = xsum; }
+    }
+    asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+    if (ctid < 4 * G) {
+        uint32_t xmax = 0;
+        float xsum = 0.f;
+        for (int w = 0; w < W; ++w) xmax = max(xmax, s_cmax[w][ctid]);
+        for (int w = 0; w < kSumThreads / 32; ++w) xsum += s_csum[w][ctid];
+        // biased exponent of the scale; a largest magnitude with an all-ones significand would round to 2^15 - 128, one
+        // more than two signed digits hold, and takes the next power of two
+        const int e = (int)(xmax >> 7) + ((xmax & 0x7fu) == 0x7fu ? 1 : 0);
+        s_xexp[ctid] = min(max(e, kP4 + 1), 254);
+        s_xsum[ctid] = xsum;
+    }
+    asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+#pragma unroll 1
+    for (int c = 0; c < 4 * G; ++c) {
+        const float mult = __uint_as_float((uint32_t)(254 + kP4 - s_xexp[c]) << 23);
+        const __nv_bfloat16* xc = x + (size_t)c * K;
+        uint4* xg = reinterpret_cast<uint4*>(xs + (size_t)(c >> 2) * group_bytes) + 8 * (c & 3);      // column blocks 2v, 2v + 1
+        for (int it = ctid; it < n_items; it += nthr) {
+            uint4* dst = xg + (size_t)(it >> 2) * (kQuadUnit / 16) + (it & 3);
+            const int k0 = k0_of(it);
+            if (k0 < K && c < B) {
+                const uint4 va = ld_x4(xc + k0), vb = ld_x4(xc + k0 + 8);
+                const uint32_t raw[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+                stage_item_quad<R>(raw, mult, dst);
+            } else {
+                dst[0] = make_uint4(0, 0, 0, 0);                  // past the end of the row, or no such vector
+                dst[4] = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
+    asm volatile("bar.sync 1, %0;" ::"r"(nthr) : "memory");
+}
+
+// One (tile, chunk) item against the G quad groups; arguments as for multiply_item_pair, every lane loads its column.
+template <int R, int G, int F0>
+__device__ __forceinline__ void multiply_item_quad(const unsigned char* wl_p, const unsigned char* wh_p, uint32_t x_sa, uint32_t xg_bytes,
+                                                   int (&acc)[kSets][4]) {
+    static_assert(R == 8 || R == 4, "quad groups serve r = 8 and r = 4");
+    constexpr int kM2 = (128 / R) / 16;
+    constexpr int kS = kSets / G;
+    const uint4 wl = *reinterpret_cast<const uint4*>(wl_p);
+    const uint4 wh = *reinterpret_cast<const uint4*>(wh_p);
+#pragma unroll
+    for (int m2 = 0; m2 < kM2; ++m2) {
+        uint4 xb[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) xb[g] = lds128(x_sa + (uint32_t)g * xg_bytes + m2 * kQuadUnit);
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+            uint32_t a0, a1, a2, a3;
+            if (R == 8) {
+                a0 = sub ? wl.z : wl.x;  a2 = sub ? wl.w : wl.y;
+                a1 = sub ? wh.z : wh.x;  a3 = sub ? wh.w : wh.y;
+            } else {
+                const int j = 2 * m2 + sub;
+                const uint32_t w_lo = j == 0 ? wl.x : j == 1 ? wl.y : j == 2 ? wl.z : wl.w;
+                const uint32_t w_hi = j == 0 ? wh.x : j == 1 ? wh.y : j == 2 ? wh.z : wh.w;
+                a0 = w_lo & 0x0f0f0f0fu;  a2 = (w_lo >> 4) & 0x0f0f0f0fu;
+                a1 = w_hi & 0x0f0f0f0fu;  a3 = (w_hi >> 4) & 0x0f0f0f0fu;
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const uint32_t b0 = sub ? xb[g].z : xb[g].x, b1 = sub ? xb[g].w : xb[g].y;
+                mma_u8s8(acc[g * kS + (F0 + 2 * m2 + sub) % kS], a0, a1, a2, a3, b0, b1);
+            }
+        }
+    }
+}
+
+template <int R, int G>
+__device__ __forceinline__ void multiply_unit_quad(const unsigned char* wl_p, const unsigned char* wh_p, uint32_t x_sa, int xq_bytes, uint32_t xg_bytes,
+                                                   int n_chunks, int (&acc)[kSets][4]) {
+    constexpr int kM2 = (128 / R) / 16;
+    constexpr int kFrag = 2 * kM2;
+    constexpr int kS = kSets / G;
+    constexpr int kU = kS > kFrag ? kS / kFrag : (R == 8 ? 2 : 1);   // as in multiply_unit_pair
+#define MATQ_QITEM(I) multiply_item_quad<R, G, ((I) * kFrag) % kS>(wl_p + (c + (I)) * 64, wh_p + (c + (I)) * 64, x_sa + (uint32_t)((c + (I)) * xq_bytes), xg_bytes, acc)
+    int c = 0;
+#pragma unroll 1
+    for (; c + kU <= n_chunks; c += kU) {
+        MATQ_QITEM(0);
+        if (kU >= 2) MATQ_QITEM(1);
+        if (kU >= 4) { MATQ_QITEM(2); MATQ_QITEM(3); }
+    }
+#pragma unroll 1
+    for (; c < n_chunks; ++c) MATQ_QITEM(0);
+#undef MATQ_QITEM
+}
+
+// Finishes one tile for the (up to four) vectors of a quad group.  Thread (g, t) holds, for rows g and g + 8, the low
+// and the high digit of vector t's sum; `yq`: y of the group's first vector, `xexp` / `xsum`: the group's entries of the
+// per-vector scale exponents and sums (shared memory), `nvec`: vectors the group really has.  Called by whole warps.
+__device__ __noinline__ void finish_tile_quad(float* __restrict__ yq, int N, int nvec, int sh, const int* xexp, const float* xsum, long long row0,
+                                              int a0, int a1, int a2, int a3, float scales, int lane, bool store) {
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int lo = h ? a2 : a0, hi = h ? a3 : a1;
+        const float al = __shfl_sync(0xffffffffu, scales, g + 8 * h), ze = __shfl_sync(0xffffffffu, scales, 16 + g + 8 * h);
+        const long long row = row0 + g + 8 * h;
+        if (t >= nvec || row >= N || !store) continue;
+        const long long tot = (long long)hi * 256 + lo;
+        const float v = __ll2float_rn(tot) * __uint_as_float((uint32_t)(xexp[t] - kP4) << 23);
+        yq[(size_t)t * N + row] = al * (v * (float)(1 << sh) - ze * xsum[t]);
+    }
+}
+
+// Q: quad groups (see above) instead of pair groups; the problems of such a launch are all at r = 8 or r = 4.
+template <int NP, int G, bool Q>
 __global__ void __launch_bounds__((kMaxW + 1) * 32, 1)
 gemv_stream_batch(const __grid_constant__ Params<NP> P) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_full[kMaxSlots], s_empty[kMaxSlots];
     __shared__ int s_tile[kTileSlots][G][16][imma::kCols];     // sums of tiles whose panels are spread over warps
     __shared__ int s_tile_cnt[kTileSlots];
-    __shared__ uint32_t s_cmax[kMaxW][kMaxBatch];
-    __shared__ float s_csum[kMaxW][kMaxBatch];
-    __shared__ int s_xexp[kMaxBatch];
-    __shared__ float s_xsum[kMaxBatch];
+    constexpr int kVec = Q ? kMaxVec : kMaxBatch;
+    __shared__ uint32_t s_cmax[kMaxW][kVec];
+    __shared__ float s_csum[kMaxW][kVec];
+    __shared__ int s_xexp[kVec];
+    __shared__ float s_xsum[kVec];
     __shared__ int s_abort;
     constexpr int kS = kSets / G;
 
@@ -349,17 +553,22 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
             first = false;
 
             const int kM2 = (128 / R) / 16;
-            const size_t group_bytes = (size_t)GE.n_qc * kM2 * kPairUnit;
-            if (R == 8) stage_activations_pair<8, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, s_cmax, s_csum, s_xexp, s_xsum);
-            else if (R == 4) stage_activations_pair<4, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, s_cmax, s_csum, s_xexp, s_xsum);
-            else stage_activations_pair<2, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, s_cmax, s_csum, s_xexp, s_xsum);
+            constexpr int kUnit = Q ? kQuadUnit : kPairUnit;
+            const size_t group_bytes = (size_t)GE.n_qc * kM2 * kUnit;
+            if constexpr (Q) {
+                if (R == 8) stage_activations_quad<8, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxVec])s_cmax, (float (*)[kMaxVec])s_csum, s_xexp, s_xsum);
+                else stage_activations_quad<4, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxVec])s_cmax, (float (*)[kMaxVec])s_csum, s_xexp, s_xsum);
+            } else if (R == 8) stage_activations_pair<8, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
+            else if (R == 4) stage_activations_pair<4, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
+            else stage_activations_pair<2, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
 
             // this lane's B source: column block g of a unit; the lanes g = 6 hold the constant column in registers
-            const int col_lane = g < kPairCols - 1 ? 1 : 0;
-            const uint32_t x_sa0 = smem_u32(xs) + (uint32_t)((g < kPairCols - 1 ? g : 0) * 4 + t) * 16u;
-            const int xq_bytes = kM2 * kPairUnit;
+            // (quad groups: every lane loads its column, there is no constant column)
+            const int col_lane = (Q || g < kPairCols - 1) ? 1 : 0;
+            const uint32_t x_sa0 = smem_u32(xs) + (uint32_t)(((Q || g < kPairCols - 1) ? g : 0) * 4 + t) * 16u;
+            const int xq_bytes = kM2 * kUnit;
             uint4 cz = make_uint4(0, 0, 0, 0);
-            if (g == kPairCols - 1) {
+            if (!Q && g == kPairCols - 1) {
                 if (R == 8) cz = make_uint4(imma::ones_b0<8>(0), imma::ones_b1<8>(0), imma::ones_b0<8>(1), imma::ones_b1<8>(1));
                 else if (R == 4) cz = make_uint4(imma::ones_b0<4>(0), imma::ones_b1<4>(0), imma::ones_b0<4>(1), imma::ones_b1<4>(1));
                 else cz = make_uint4(imma::ones_b0<2>(0), imma::ones_b1<2>(0), imma::ones_b0<2>(1), imma::ones_b1<2>(1));
@@ -371,7 +580,10 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
                 const unsigned char* wl_p = base + (size_t)g * GE.stride;
                 const unsigned char* wh_p = base + (size_t)(g + 8) * GE.stride;
                 const uint32_t x_sa = x_sa0 + (uint32_t)(q0 * xq_bytes);
-                if (R == 8) multiply_unit_pair<8, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, col_lane, cz, q1 - q0, acc);
+                if constexpr (Q) {
+                    if (R == 8) multiply_unit_quad<8, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, q1 - q0, acc);
+                    else multiply_unit_quad<4, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, q1 - q0, acc);
+                } else if (R == 8) multiply_unit_pair<8, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, col_lane, cz, q1 - q0, acc);
                 else if (R == 4) multiply_unit_pair<4, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, col_lane, cz, q1 - q0, acc);
                 else multiply_unit_pair<2, G>(wl_p, wh_p, x_sa, xq_bytes, (uint32_t)group_bytes, col_lane, cz, q1 - q0, acc);
             };
@@ -397,6 +609,15 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
                 float scales = 0.f;
                 if (row < pr.N) scales = lane < 16 ? pr.alpha[row] : pr.zero[row];
                 const bool store = !*abort_flag;
+                if constexpr (Q) {
+#pragma unroll
+                    for (int gg = 0; gg < G; ++gg) {
+                        if (4 * gg >= B) break;
+                        finish_tile_quad(pr.y + (size_t)(4 * gg) * pr.N, pr.N, min(4, B - 4 * gg), sh, s_xexp + 4 * gg, s_xsum + 4 * gg, row0,
+                                         acc[gg * kS][0], acc[gg * kS][1], acc[gg * kS][2], acc[gg * kS][3], scales, lane, store);
+                    }
+                    return;
+                }
 #pragma unroll
                 for (int gg = 0; gg < G; ++gg) {
                     if (2 * gg >= B) break;
@@ -417,7 +638,7 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
                 for (int gg = 0; gg < G; ++gg) {
                     atomicAdd(&s_tile[ts][gg][g][2 * t], acc[gg * kS][0]);
                     atomicAdd(&s_tile[ts][gg][g + 8][2 * t], acc[gg * kS][2]);
-                    if (t < 3) { atomicAdd(&s_tile[ts][gg][g][2 * t + 1], acc[gg * kS][1]); atomicAdd(&s_tile[ts][gg][g + 8][2 * t + 1], acc[gg * kS][3]); }
+                    if (Q || t < 3) { atomicAdd(&s_tile[ts][gg][g][2 * t + 1], acc[gg * kS][1]); atomicAdd(&s_tile[ts][gg][g + 8][2 * t + 1], acc[gg * kS][3]); }
                 }
                 __threadfence_block();
                 __syncwarp();
@@ -496,23 +717,28 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
 // ---------------------------------------------------------------------------------------------------------------
 // Host side
 
-inline int groups_of(int64_t B) { return B <= 2 ? 1 : B <= 4 ? 2 : 4; }
-
 // static shared memory of the batched kernel with G groups, rounded up
 inline int static_reserve_batch(int G) { return (10 + (G - 1) * 6) * 1024; }
 
+// Quad groups (four vectors a group, 15-bit activations) serve r = 8 and r = 4 from three vectors up; pair groups (two
+// vectors a group, 22-bit activations) everything else.
+inline bool quad_mode(int r, int64_t B) { return r != 2 && B >= 3; }
+inline int groups_of(int64_t B, bool quad) { return quad ? (B <= 4 ? 1 : B <= 8 ? 2 : 4) : (B <= 2 ? 1 : B <= 4 ? 2 : 4); }
+inline long long batch_fit(const Geo& g, int r, int G, bool quad) {
+    return ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, r, quad))) / slot_bytes_of(g);
+}
+
 // Whether a problem with B vectors (2 <= B <= kMaxBatch) can take the batched path.
 inline bool eligible_batch(int64_t N, int64_t K, int r, int64_t B) {
-    if (B < 2 || B > kMaxBatch) return false;
+    const bool quad = quad_mode(r, B);
+    if (B < 2 || B > (quad ? kMaxVec : kMaxBatch)) return false;
     if (!(r == 8 || r == 4 || r == 2) || K % 128 != 0 || (r == 2 && K % 256 != 0) || K > imma::kMaxK || N <= 0 || N >= (1ll << 31) - 16) return false;
     const Geo g = geometry((int)N, (int)K, r, kUnitRow);
-    const int G = groups_of(B);
-    const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, r))) / slot_bytes_of(g);
-    return fit >= kMinW;
+    return batch_fit(g, r, groups_of(B, quad), quad) >= kMinW;
 }
 
 // One launch over a list of problems that all take the batched path (hb[i]: the vectors of problem i).
-template <int NP, int G>
+template <int NP, int G, bool Q>
 inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     static std::atomic<unsigned long long> smem_ok{0};
     Params<NP> P;
@@ -540,7 +766,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
         const Geo g = geometry(q.N, q.K, q.r, kUnitRow);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
         item0 += (long long)g.tiles * tile_cost(g, q.r);
-        xs_bytes = std::max(xs_bytes, (size_t)G * xs_group_bytes_of(g, q.r));
+        xs_bytes = std::max(xs_bytes, (size_t)G * xs_group_bytes_of(g, q.r, Q));
         slot_bytes = std::max(slot_bytes, slot_bytes_of(g));
         ++m;
     }
@@ -554,7 +780,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     const int slots = fit / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = kUnitRow; P.hold = hold ? 1 : 0; P.pairs = 0;
-    auto kern = gemv_stream_batch<NP, G>;
+    auto kern = gemv_stream_batch<NP, G, Q>;
     if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
@@ -571,20 +797,23 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
 }
 
 template <int NP>
-inline int launch_list_batch_g(int G, const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
-    if (G == 1) return launch_list_batch<NP, 1>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-    if (G == 2) return launch_list_batch<NP, 2>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-    return launch_list_batch<NP, 4>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+inline int launch_list_batch_g(int G, bool quad, const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
+    if (quad) {
+        if (G == 1) return launch_list_batch<NP, 1, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+        if (G == 2) return launch_list_batch<NP, 2, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+        return launch_list_batch<NP, 4, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+    }
+    if (G == 1) return launch_list_batch<NP, 1, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+    if (G == 2) return launch_list_batch<NP, 2, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+    return launch_list_batch<NP, 4, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
 }
 
 // The largest number of column groups (4, 2 or 1) whose staged activations leave room for at least kMinW stages; 0 when
 // not even one group fits.
-inline int max_groups(int64_t N, int64_t K, int r) {
+inline int max_groups(int64_t N, int64_t K, int r, bool quad) {
     const Geo g = geometry((int)N, (int)K, r, kUnitRow);
-    for (int G = 4; G >= 1; G /= 2) {
-        const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, r))) / slot_bytes_of(g);
-        if (fit >= kMinW) return G;
-    }
+    for (int G = 4; G >= 1; G /= 2)
+        if (batch_fit(g, r, G, quad) >= kMinW) return G;
     return 0;
 }
 
@@ -598,20 +827,20 @@ inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, l
     // property of the launch, and the short rows of a stack should not run with four.
     std::vector<HostProblem> sel;
     std::vector<int> sel_b;
+    for (int quad = 0; quad < 2; ++quad)
     for (int G = 1; G <= 4; G *= 2)
         for (int wide = 0; wide < 2; ++wide) {
             sel.clear(); sel_b.clear();
             for (int i = 0; i < n; ++i) {
-                if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
+                if (hp[i].N == 0 || quad_mode(hp[i].r, hb[i]) != (quad == 1) || groups_of(hb[i], quad == 1) != G) continue;
                 const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-                const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
-                if ((fit >= kWideFit) != (wide == 0)) continue;
+                if ((batch_fit(g, hp[i].r, G, quad == 1) >= kWideFit) != (wide == 0)) continue;
                 sel.push_back(hp[i]); sel_b.push_back(hb[i]);
             }
             for (size_t i = 0; i < sel.size(); i += kLargeList) {
                 const int cnt = (int)std::min<size_t>(kLargeList, sel.size() - i);
-                const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s)
-                                                 : launch_list_batch_g<kLargeList>(G, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s);
+                const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s)
+                                                 : launch_list_batch_g<kLargeList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s);
                 if (st != MATQ_OK) return st;
             }
         }
@@ -621,14 +850,14 @@ inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, l
 // Number of launches launch_batch makes for these batch sizes and shapes.
 inline int count_batch_launches(const HostProblem* hp, const int* hb, int n) {
     int launches = 0;
+    for (int quad = 0; quad < 2; ++quad)
     for (int G = 1; G <= 4; G *= 2)
         for (int wide = 0; wide < 2; ++wide) {
             size_t cnt = 0;
             for (int i = 0; i < n; ++i) {
-                if (hp[i].N == 0 || groups_of(hb[i]) != G) continue;
+                if (hp[i].N == 0 || quad_mode(hp[i].r, hb[i]) != (quad == 1) || groups_of(hb[i], quad == 1) != G) continue;
                 const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-                const long long fit = ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, hp[i].r))) / slot_bytes_of(g);
-                cnt += (fit >= kWideFit) == (wide == 0);
+                cnt += (batch_fit(g, hp[i].r, G, quad == 1) >= kWideFit) == (wide == 0);
             }
             launches += (int)((cnt + kLargeList - 1) / kLargeList);
         }
@@ -639,9 +868,10 @@ inline int count_batch_launches(const HostProblem* hp, const int* hb, int n) {
 // the plane (`many`, with their sizes in `many_b`), a single left-over vector as a problem of its own (`one`).
 inline int split_batch(const HostProblem& q, std::vector<HostProblem>& one, std::vector<HostProblem>& many, std::vector<int>& many_b) {
     if (q.N == 0) return MATQ_OK;
-    const int Gmax = max_groups(q.N, q.K, q.r);
+    const bool quad = quad_mode(q.r, q.B);
+    const int Gmax = max_groups(q.N, q.K, q.r, quad);
     if (Gmax == 0) return MATQ_ERR_SHAPE;
-    const int64_t step = std::min<int64_t>(2 * Gmax, kMaxBatch);
+    const int64_t step = quad ? std::min<int64_t>(4 * Gmax, kMaxVec) : std::min<int64_t>(2 * Gmax, kMaxBatch);
     for (int64_t b0 = 0; b0 < q.B; b0 += step) {
         HostProblem part = q;
         const int64_t nb = std::min<int64_t>(step, q.B - b0);

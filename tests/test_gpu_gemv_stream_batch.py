@@ -1,11 +1,14 @@
 """GPU parity of the batched persistent decode GEMV (2 <= B <= 16 activation vectors per problem: MATQ_GEMV_STREAM
 with B > 1, and matq_gemv_grouped with batches) against the CPU oracle.
 
-The weights' sums are exact integers.  An activation is a 22-bit integer relative to the largest magnitude of its
-vector, and a field that sits s bits up in its byte meets its activation divided by 2^s, so the activations of the top
-field keep 22 - (8 - r) bits: rounding steps of 2^-22 (r = 8), 2^-18 (r = 4) and 2^-16 (r = 2) of 2 max|x|.  With
-max|x| / rms(x) about 4 that is 1e-6, 2e-5 and 6e-5 of rms(y); the tests allow 1e-4, 3e-4 and 1e-3 (the bf16 tensor
-path for batches is held to 1e-2).
+The weights' sums are exact integers.  Two vectors, and every batch at r = 2 (pair groups): an activation is a 22-bit
+integer relative to the largest magnitude of its vector, and a field that sits s bits up in its byte meets its
+activation divided by 2^s, so the activations of the top field keep 22 - (8 - r) bits: rounding steps of 2^-22 (r = 8),
+2^-18 (r = 4) and 2^-16 (r = 2) of 2 max|x|.  With max|x| / rms(x) about 4 that is 1e-6, 2e-5 and 6e-5 of rms(y); the
+tests allow 1e-4, 3e-4 and 1e-3.  Three or more vectors at r = 8 and r = 4 (quad groups): a 15-bit integer and its sign,
+a rounding step of 2^-14 (2^-13 when the largest magnitude's significand is all ones) of the power of two at or below
+max|x|, the same for both fields: about 4e-5 of rms(y) per output, 2e-4 at worst over tens of thousands of outputs; the
+tests allow 1e-3 (the bound for the tensor-core paths is 1e-2 rms(y); the bf16 tensor path for batches is held to that).
 """
 import numpy as np
 import pytest
@@ -19,6 +22,11 @@ from tests.util import bf16_dev, dev, host, rms, status_word
 pytestmark = pytest.mark.gpu
 
 TOL = {8: 1e-4, 4: 3e-4, 2: 1e-3}
+TOL_QUAD = 1e-3
+
+
+def tol(r, B):
+    return TOL_QUAD if (r != 2 and B >= 3) else TOL[r]
 
 
 def _problem(N, K, r, B, seed, scales=None):
@@ -37,7 +45,7 @@ def _problem(N, K, r, B, seed, scales=None):
 def _check(y, y_ref, r):
     y = host(y).reshape(y_ref.shape)
     for b in range(y_ref.shape[0]):
-        assert np.abs(y[b] - y_ref[b]).max() <= TOL[r] * rms(y_ref[b]), f"vector {b}"
+        assert np.abs(y[b] - y_ref[b]).max() <= tol(r, y_ref.shape[0]) * rms(y_ref[b]), f"vector {b}"
 
 
 @pytest.mark.parametrize("r", [8, 4, 2])
@@ -57,7 +65,7 @@ def test_stream_batch_single_problem(r, B, N, K):
 
 @pytest.mark.parametrize("r", [8, 4, 2])
 def test_stream_batch_sixteen_vectors(r):
-    # more than 8 vectors: two problems of 8 that share the plane
+    # sixteen vectors: one problem of four quad groups at r = 8 and 4, two problems of 8 that share the plane at r = 2
     p = _problem(700, 2304, r, 16, 7100 + r)
     y = mq.gemv(dev(p["packed"]), 2304, r, dev(p["a"]), dev(p["z"]), bf16_dev(p["x"]), flags=mq.GEMV_STREAM)
     _check(y, p["y_ref"], p["r"])
@@ -72,7 +80,7 @@ def test_stream_batch_vectors_of_different_magnitude(r):
     y = host(y)
     for b in range(6):
         ref_b = p["y_ref"][b]
-        assert np.abs(y[b] - ref_b).max() <= TOL[r] * max(rms(ref_b), 1e-30), f"vector {b}"
+        assert np.abs(y[b] - ref_b).max() <= tol(r, 6) * max(rms(ref_b), 1e-30), f"vector {b}"
 
 
 def test_stream_batch_exact_integers():
