@@ -243,9 +243,19 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, volati
     }
 }
 
-// The next problem (from index p on) of which this CTA owns tiles, and which: [t_lo, t_hi).
+// The next problem (from index p on) of which this CTA owns tiles, and which: [t_lo, t_hi).  A share of rows with
+// several K panels that is not a whole number of rounds (W groups of tiles, one per warp) comes as two segments: the
+// whole rounds, which the warps take a tile each, and the rest (`tail_lo`, `tail_hi`: state of the iteration, -1 = none),
+// fewer groups than warps, whose panels plan_of() spreads over all warps; otherwise the last round would keep a few
+// warps busy for a whole tile (K = 9216 at r = 8: 147 KB) while the others idle.  Problem p - 1 is the current one for
+// both segments.
 template <int NP>
-__device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, long long hi, int& p, int& t_lo, int& t_hi) {
+__device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, long long hi, int& p, int& t_lo, int& t_hi, int& tail_lo, int& tail_hi) {
+    if (tail_lo >= 0) {
+        t_lo = tail_lo; t_hi = tail_hi;
+        tail_lo = -1;
+        return true;
+    }
     while (p < P.n) {
         const long long i0 = P.p[p].item0;
         if (i0 >= hi) return false;
@@ -256,7 +266,16 @@ __device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, 
         ++p;
         t_lo = (int)(a < g.tiles ? a : g.tiles);
         t_hi = (int)(b < g.tiles ? b : g.tiles);
-        if (t_lo < t_hi) return true;
+        if (t_lo < t_hi) {
+            if (g.n_panels > 1) {
+                const int Tu = (t_hi - t_lo + g.tpu - 1) / g.tpu, rem = Tu % P.W;
+                if (Tu > P.W && rem != 0 && rem <= P.W - 2) {
+                    tail_lo = t_lo + (Tu - rem) * g.tpu; tail_hi = t_hi;
+                    t_hi = tail_lo;
+                }
+            }
+            return true;
+        }
     }
     return false;
 }
@@ -725,10 +744,10 @@ __device__ __forceinline__ void producer_warp(const Params<NP>& P, long long lo,
     // ------------------------------------------------------------------ producer warp: lane l < W feeds warp l's stages
     int it0 = 0;                                          // units of the segments before this one (a multiple of W)
     bool waited = P.pdl != 1;
-    int p = p_first, t_lo, t_hi;
+    int p = p_first, t_lo, t_hi, tail_lo = -1, tail_hi = 0;
     bool ok = true;
     int last_it = -1;                                     // latest unit this lane issued a copy for
-    while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi)) {
+    while (ok && !P.hold && next_segment(P, lo, hi, p, t_lo, t_hi, tail_lo, tail_hi)) {
         const Problem& pr = P.p[p - 1];
         const Geo G = geometry(pr.N, pr.K, pr.r, P.unit_row, P.pairs);
         const int T = t_hi - t_lo;
@@ -860,13 +879,13 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
         const int ctid = tid;                                  // warps 0 .. W-1
         int it0 = 0;                                           // units of the segments before this one (a multiple of W)
         int split_tiles = 0;                                   // split-mode tiles of earlier segments (a tile's slot = its count mod kTileSlots)
-        int p = p_first, t_lo, t_hi;
+        int p = p_first, t_lo, t_hi, tail_lo = -1, tail_hi = 0, staged_p = -1;
         bool first = true;
         bool ep_ready = P.pdl != 2;                            // whether ep_rowsum's sums may be read yet
         Geo G;
         float xsum = 0.f;
         int xexp = 0;
-        while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
+        while (next_segment(P, lo, hi, p, t_lo, t_hi, tail_lo, tail_hi)) {
             const Problem& pr = P.p[p - 1];
             G = geometry(pr.N, pr.K, pr.r, P.unit_row, P.pairs);
             const int R = RF ? RF : pr.r;
@@ -892,9 +911,12 @@ gemv_stream(const __grid_constant__ Params<NP> P) {
             first = false;
 
             // ---- the activations of this problem as byte units in fragment order (all consumer warps together)
-            if (R == 8) stage_activations<8>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
+            // (the second segment of a problem finds them staged)
+            if (staged_p == p) {}
+            else if (R == 8) stage_activations<8>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
             else if (R == 4) stage_activations<4>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
             else stage_activations<2>(pr.x, pr.K, G.n_qc, xs, ctid, nthr, W, s_rmax, s_rsum, xsum, xexp);
+            staged_p = p;
 
             const int kM2 = (128 / R) / 16;
             // this lane's B source: chunk q of byte column g starts at xs[q * kM2 * 16 + g * 4 + t]; the lanes g = 4 hold

@@ -528,9 +528,9 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
         const int g = lane >> 2, t = lane & 3;
         const int ctid = tid;
         int it0 = 0, split_tiles = 0;
-        int p = p_first, t_lo, t_hi;
+        int p = p_first, t_lo, t_hi, tail_lo = -1, tail_hi = 0, staged_p = -1;
         bool first = true;
-        while (next_segment(P, lo, hi, p, t_lo, t_hi)) {
+        while (next_segment(P, lo, hi, p, t_lo, t_hi, tail_lo, tail_hi)) {
             const Problem& pr = P.p[p - 1];
             const Geo GE = geometry(pr.N, pr.K, pr.r, P.unit_row);
             const int R = pr.r;
@@ -555,12 +555,14 @@ gemv_stream_batch(const __grid_constant__ Params<NP> P) {
             const int kM2 = (128 / R) / 16;
             constexpr int kUnit = Q ? kQuadUnit : kPairUnit;
             const size_t group_bytes = (size_t)GE.n_qc * kM2 * kUnit;
-            if constexpr (Q) {
+            if (staged_p == p) {                                  // the second segment of a problem finds them staged
+            } else if constexpr (Q) {
                 if (R == 8) stage_activations_quad<8, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxVec])s_cmax, (float (*)[kMaxVec])s_csum, s_xexp, s_xsum);
                 else stage_activations_quad<4, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxVec])s_cmax, (float (*)[kMaxVec])s_csum, s_xexp, s_xsum);
             } else if (R == 8) stage_activations_pair<8, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
             else if (R == 4) stage_activations_pair<4, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
             else stage_activations_pair<2, G>(pr.x, pr.K, B, GE.n_qc, xs, group_bytes, ctid, nthr, W, (uint32_t (*)[kMaxBatch])s_cmax, (float (*)[kMaxBatch])s_csum, s_xexp, s_xsum);
+            staged_p = p;
 
             // this lane's B source: column block g of a unit; the lanes g = 6 hold the constant column in registers
             // (quad groups: every lane loads its column, there is no constant column)
@@ -727,25 +729,32 @@ inline int groups_of(int64_t B, bool quad) { return quad ? (B <= 4 ? 1 : B <= 8 
 inline long long batch_fit(const Geo& g, int r, int G, bool quad) {
     return ((long long)kSmemLimit - static_reserve_batch(G) - (long long)(G * xs_group_bytes_of(g, r, quad))) / slot_bytes_of(g);
 }
+// Stages a problem gets beside its staged activations.  Long rows leave few stages of the usual size (K = 9216, eight
+// vectors: four); such problems run in launches of their own with units half as large (`narrow`), i.e. with twice
+// the stages and warps.
+inline long long batch_fit(int64_t N, int64_t K, int r, int G, bool quad, bool* narrow = nullptr) {
+    const long long full = batch_fit(geometry((int)N, (int)K, r, kUnitRow), r, G, quad);
+    if (narrow) *narrow = full < kWideFit;
+    return full >= kWideFit ? full : batch_fit(geometry((int)N, (int)K, r, kUnitRow / 2), r, G, quad);
+}
 
 // Whether a problem with B vectors (2 <= B <= kMaxBatch) can take the batched path.
 inline bool eligible_batch(int64_t N, int64_t K, int r, int64_t B) {
     const bool quad = quad_mode(r, B);
     if (B < 2 || B > (quad ? kMaxVec : kMaxBatch)) return false;
     if (!(r == 8 || r == 4 || r == 2) || K % 128 != 0 || (r == 2 && K % 256 != 0) || K > imma::kMaxK || N <= 0 || N >= (1ll << 31) - 16) return false;
-    const Geo g = geometry((int)N, (int)K, r, kUnitRow);
-    return batch_fit(g, r, groups_of(B, quad), quad) >= kMinW;
+    return batch_fit(N, K, r, groups_of(B, quad), quad) >= kMinW;
 }
 
 // One launch over a list of problems that all take the batched path (hb[i]: the vectors of problem i).
 template <int NP, int G, bool Q>
-inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
+inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, int unit_row, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     static std::atomic<unsigned long long> smem_ok{0};
     Params<NP> P;
     long long items = 0, tiles = 0;
     for (int i = 0; i < n; ++i) {
         if (hp[i].N == 0) continue;
-        const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
+        const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, unit_row);
         items += (long long)g.tiles * tile_cost(g, hp[i].r);
         tiles += g.tiles;
     }
@@ -763,7 +772,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
         q.x = static_cast<const __nv_bfloat16*>(hp[i].x); q.y = hp[i].y;
         q.N = (int)hp[i].N; q.K = (int)hp[i].K; q.r = hp[i].r; q.B = hb[i];
         q.item0 = item0;
-        const Geo g = geometry(q.N, q.K, q.r, kUnitRow);
+        const Geo g = geometry(q.N, q.K, q.r, unit_row);
         if (!g.contig && !make_plane_map(&P.tm[m], q.packed, q.N, g)) return MATQ_ERR_CUDA;
         item0 += (long long)g.tiles * tile_cost(g, q.r);
         xs_bytes = std::max(xs_bytes, (size_t)G * xs_group_bytes_of(g, q.r, Q));
@@ -779,7 +788,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
     W = pick_warps(W, fit);
     const int slots = fit / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
-    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = kUnitRow; P.hold = hold ? 1 : 0; P.pairs = 0;
+    P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0; P.pairs = 0;
     auto kern = gemv_stream_batch<NP, G, Q>;
     if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -797,23 +806,22 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, bool p
 }
 
 template <int NP>
-inline int launch_list_batch_g(int G, bool quad, const HostProblem* hp, const int* hb, int n, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
+inline int launch_list_batch_g(int G, bool quad, const HostProblem* hp, const int* hb, int n, int unit_row, bool pdl, long long wait_cycles, bool hold, int32_t* dev_status, cudaStream_t s) {
     if (quad) {
-        if (G == 1) return launch_list_batch<NP, 1, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-        if (G == 2) return launch_list_batch<NP, 2, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-        return launch_list_batch<NP, 4, true>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+        if (G == 1) return launch_list_batch<NP, 1, true>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
+        if (G == 2) return launch_list_batch<NP, 2, true>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
+        return launch_list_batch<NP, 4, true>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
     }
-    if (G == 1) return launch_list_batch<NP, 1, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-    if (G == 2) return launch_list_batch<NP, 2, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
-    return launch_list_batch<NP, 4, false>(hp, hb, n, pdl, wait_cycles, hold, dev_status, s);
+    if (G == 1) return launch_list_batch<NP, 1, false>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
+    if (G == 2) return launch_list_batch<NP, 2, false>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
+    return launch_list_batch<NP, 4, false>(hp, hb, n, unit_row, pdl, wait_cycles, hold, dev_status, s);
 }
 
 // The largest number of column groups (4, 2 or 1) whose staged activations leave room for at least kMinW stages; 0 when
 // not even one group fits.
 inline int max_groups(int64_t N, int64_t K, int r, bool quad) {
-    const Geo g = geometry((int)N, (int)K, r, kUnitRow);
     for (int G = 4; G >= 1; G /= 2)
-        if (batch_fit(g, r, G, quad) >= kMinW) return G;
+        if (batch_fit(N, K, r, G, quad) >= kMinW) return G;
     return 0;
 }
 
@@ -833,14 +841,15 @@ inline int launch_batch(const HostProblem* hp, const int* hb, int n, bool pdl, l
             sel.clear(); sel_b.clear();
             for (int i = 0; i < n; ++i) {
                 if (hp[i].N == 0 || quad_mode(hp[i].r, hb[i]) != (quad == 1) || groups_of(hb[i], quad == 1) != G) continue;
-                const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-                if ((batch_fit(g, hp[i].r, G, quad == 1) >= kWideFit) != (wide == 0)) continue;
+                bool narrow = false;
+                batch_fit(hp[i].N, hp[i].K, hp[i].r, G, quad == 1, &narrow);
+                if (narrow != (wide == 1)) continue;
                 sel.push_back(hp[i]); sel_b.push_back(hb[i]);
             }
             for (size_t i = 0; i < sel.size(); i += kLargeList) {
                 const int cnt = (int)std::min<size_t>(kLargeList, sel.size() - i);
-                const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s)
-                                                 : launch_list_batch_g<kLargeList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, pdl, wait_cycles, hold, dev_status, s);
+                const int st = cnt <= kSmallList ? launch_list_batch_g<kSmallList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, wide ? kUnitRow / 2 : kUnitRow, pdl, wait_cycles, hold, dev_status, s)
+                                                 : launch_list_batch_g<kLargeList>(G, quad == 1, sel.data() + i, sel_b.data() + i, cnt, wide ? kUnitRow / 2 : kUnitRow, pdl, wait_cycles, hold, dev_status, s);
                 if (st != MATQ_OK) return st;
             }
         }
@@ -856,8 +865,9 @@ inline int count_batch_launches(const HostProblem* hp, const int* hb, int n) {
             size_t cnt = 0;
             for (int i = 0; i < n; ++i) {
                 if (hp[i].N == 0 || quad_mode(hp[i].r, hb[i]) != (quad == 1) || groups_of(hb[i], quad == 1) != G) continue;
-                const Geo g = geometry((int)hp[i].N, (int)hp[i].K, hp[i].r, kUnitRow);
-                cnt += (batch_fit(g, hp[i].r, G, quad == 1) >= kWideFit) == (wide == 0);
+                bool narrow = false;
+                batch_fit(hp[i].N, hp[i].K, hp[i].r, G, quad == 1, &narrow);
+                cnt += narrow == (wide == 1);
             }
             launches += (int)((cnt + kLargeList - 1) / kLargeList);
         }
