@@ -52,7 +52,7 @@ METRIC = "sliced int{8,4,2} GEMV HBM GB/s (% of peak); multi-precision GEMM TFLO
 NCU = {
     # matq_gemv_grouped on 12 matrices of this stack (profiles/gemv_stream_*.md): DRAM bytes / algorithmic bytes
     "gemv_stream_ratio_r4": 1.022,
-    "gemv_stream_ratio_r2": 0.991,
+    "gemv_stream_ratio_r2": 0.992,
     "quantize": 42780000,
 }
 CONFIG_ID = 2

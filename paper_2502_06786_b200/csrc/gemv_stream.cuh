@@ -120,6 +120,7 @@ struct Params {
     int W;                    // consumer warps
     int pdl;                  // 0: plain launch; 1: programmatic dependent of an unknown kernel (wait before x is read);
                               // 2: dependent of ep_rowsum, released after that kernel's own wait (wait before its sums are read)
+    int tails;                // whether a share that is not a whole number of rounds is cut in two (see next_segment)
     int unit_row;             // bytes per row of the largest unit
     int hold;                 // diagnostics: the producer issues no copies, so every wait for a stage runs out
     int pairs;                // geometry with an even number of tiles per unit (see geometry())
@@ -267,7 +268,7 @@ __device__ __forceinline__ bool next_segment(const Params<NP>& P, long long lo, 
         t_lo = (int)(a < g.tiles ? a : g.tiles);
         t_hi = (int)(b < g.tiles ? b : g.tiles);
         if (t_lo < t_hi) {
-            if (g.n_panels > 1) {
+            if (P.tails && g.n_panels > 1) {
                 const int Tu = (t_hi - t_lo + g.tpu - 1) / g.tpu, rem = Tu % P.W;
                 if (Tu > P.W && rem != 0 && rem <= P.W - 2) {
                     tail_lo = t_lo + (Tu - rem) * g.tpu; tail_hi = t_hi;
@@ -1302,6 +1303,7 @@ inline int launch_list(const HostProblem* hp, int n, bool pdl, long long wait_cy
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = behind_ep ? 2 : pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0;
     P.pairs = pairs;
+    P.tails = 1;
     auto kern = behind_ep ? (rf == 8 ? gemv_stream<NP, 8, true> : rf == 4 ? gemv_stream<NP, 4, true> : rf == 2 ? gemv_stream<NP, 2, true> : gemv_stream<NP, 0, true>)
                           : (rf == 8 ? gemv_stream<NP, 8, false> : rf == 4 ? gemv_stream<NP, 4, false> : rf == 2 ? gemv_stream<NP, 2, false> : gemv_stream<NP, 0, false>);
     if (!opt_in_max_smem(kern, smem_ok[(behind_ep ? 4 : 0) + (rf == 8 ? 3 : rf == 4 ? 2 : rf == 2 ? 1 : 0)])) return MATQ_ERR_CUDA;

@@ -789,6 +789,7 @@ inline int launch_list_batch(const HostProblem* hp, const int* hb, int n, int un
     const int slots = fit / W * W;
     P.items = items; P.wait_cycles = wait_cycles; P.dev_status = dev_status; P.n = m; P.slots = slots; P.slot_bytes = slot_bytes;
     P.xs_bytes = (int)xs_bytes; P.W = W; P.pdl = pdl ? 1 : 0; P.unit_row = unit_row; P.hold = hold ? 1 : 0; P.pairs = 0;
+    P.tails = 1;
     auto kern = gemv_stream_batch<NP, G, Q>;
     if (!opt_in_max_smem(kern, smem_ok)) return MATQ_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -820,6 +821,10 @@ inline int launch_list_batch_g(int G, bool quad, const HostProblem* hp, const in
 // The largest number of column groups (4, 2 or 1) whose staged activations leave room for at least kMinW stages; 0 when
 // not even one group fits.
 inline int max_groups(int64_t N, int64_t K, int r, bool quad) {
+    // more groups only while they leave at least six stages (and warps): K = 14336 at r = 2 takes two vectors with seven
+    // stages twice rather than four with four stages once
+    for (int G = 4; G >= 1; G /= 2)
+        if (batch_fit(N, K, r, G, quad) >= kWideFit - 1) return G;
     for (int G = 4; G >= 1; G /= 2)
         if (batch_fit(N, K, r, G, quad) >= kMinW) return G;
     return 0;
