@@ -26,7 +26,11 @@
 //
 // Not here: extra-precision lists with B > 1 (those calls keep the bf16 kernel of gemv_tensor.cuh), r = 2 planes
 // whose K is not a multiple of 256.  Batches above 8, or above what the staged activations of a long row leave room
-// for (K = 9216: four vectors), are cut into problems that share the plane; the later ones find it in the L2.
+// for, are cut into problems that share the plane; the later ones find it in the L2.
+//
+// Quad groups.  At r = 8 and r = 4, batches of three or more vectors use a second column layout (further down): four
+// vectors per group as two signed digits each, a u8 x s8 MMA, no constant column; half the MMAs and fragment loads
+// for the same vectors, up to 16 vectors per problem, 15-bit activations instead of 22-bit ones.
 #pragma once
 #include <vector>
 
